@@ -1,0 +1,203 @@
+/*
+ * lava.h -- C ABI of the LAVa prefill-time KV-cache eviction hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library scores every cached (KV head, position) entry of a layer with the LAVa metric,
+ * turns per-layer score entropies into integer layer budgets, selects the layer-wide top-k
+ * (which yields per-head budgets) and gathers the retained K/V rows into a packed cache.
+ *
+ * Conventions that hold for every function unless its comment says otherwise:
+ *   - Every data pointer is a caller-owned DEVICE pointer.  The library never allocates or
+ *     frees device memory and never synchronises the device; all work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*, NULL = the legacy default stream).
+ *   - Pointers must be 16-byte aligned, token rows contiguous (`head_dim` elements), strides
+ *     are in elements and multiples of 8.
+ *   - Functions return a lava_status.  Arguments are validated on the host before any launch;
+ *     on error nothing is enqueued and lava_last_error() describes the problem.  No C++
+ *     exception crosses this boundary.
+ *   - Failures that only the device can see (a sequence shorter than the window, an
+ *     infeasible budget, an expired bounded wait) set bits in the status word at the start
+ *     of the workspace; read it with lava_poll_status().
+ *
+ * Positions are 0-based.  For a sequence of n tokens and window w, P = n - w is the number of
+ * prefix candidates; the window is positions P..n-1 and is always retained (constraints of
+ * Eq. 1).  "Head" in budgets and offsets means KV head.
+ *
+ * Score layout (one layer):  sequence b, KV head g, prefix position i lives at
+ *      H_kv * (cu_seqlens[b] - b*w)  +  g * P_b  +  i
+ * so one sequence's scores form one contiguous flat array of H_kv*P_b floats, heads in order.
+ * A layer has  total_scores = H_kv * (total_tokens - batch*w)  entries.
+ */
+#ifndef LAVA_H_
+#define LAVA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LAVA_API __attribute__((visibility("default")))
+#else
+#define LAVA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lava_status {
+  LAVA_OK = 0,
+  LAVA_ERR_INVALID_ARG = 1,  /* null / misaligned pointer, bad geometry */
+  LAVA_ERR_UNSUPPORTED = 2,  /* valid request outside what the kernels cover */
+  LAVA_ERR_WORKSPACE = 3,    /* workspace missing or smaller than lava_workspace_bytes() */
+  LAVA_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed */
+  LAVA_ERR_TIMEOUT = 5       /* a bounded device-side wait expired (reported by poll) */
+} lava_status;
+
+typedef enum lava_dtype { LAVA_F32 = 0, LAVA_BF16 = 1 } lava_dtype;
+typedef enum lava_pool { LAVA_POOL_NONE = 0, LAVA_POOL_MAX = 1, LAVA_POOL_AVG = 2 } lava_pool;
+typedef enum lava_budget_mode { LAVA_BUDGET_DYNAMIC = 0, LAVA_BUDGET_UNIFORM = 1 } lava_budget_mode;
+
+/* Bits of the device status word. */
+#define LAVA_DEV_SHORT_SEQUENCE 1u    /* some sequence has fewer than `window` tokens        */
+#define LAVA_DEV_BUDGET_INFEASIBLE 2u /* total budget outside [L*floor, L*cap]; was clamped  */
+#define LAVA_DEV_WAIT_EXPIRED 4u      /* a bounded wait inside a kernel gave up              */
+
+/* Geometry of one layer (all layers of a model share it).  Plain data, caller-owned (host). */
+typedef struct lava_layer_desc {
+  int32_t n_q_heads;   /* H_q, a multiple of n_kv_heads                                     */
+  int32_t n_kv_heads;  /* H_kv                                                              */
+  int32_t head_dim;    /* d_h: 64 or 128                                                    */
+  int32_t window;      /* w >= 1: observation window = last w tokens of each sequence       */
+  int32_t pool_kind;   /* lava_pool                                                         */
+  int32_t pool_kernel; /* odd, 1..63; ignored for LAVA_POOL_NONE                            */
+  int32_t dtype;       /* lava_dtype of Q, K, V and of the compacted output                 */
+  int32_t batch;       /* number of sequences (>= 1)                                        */
+  int32_t max_seqlen;  /* upper bound on any sequence length (0 => total_tokens)            */
+  int32_t reserved;    /* must be 0                                                         */
+  const int32_t* cu_seqlens; /* device int32 [batch+1] token offsets; NULL => batch == 1    */
+  int64_t total_tokens;      /* sum of sequence lengths                                     */
+  int64_t k_stride_head, k_stride_tok; /* K[g][tok][c] = k[g*k_stride_head + tok*k_stride_tok + c] */
+  int64_t v_stride_head, v_stride_tok;
+  float sm_scale;      /* logit scale; 0 => 1/sqrt(head_dim)                                */
+  float c_hat;         /* optional ||W_O^T||_1 factor of Theorem 1; 0 => 1.  Multiplies every
+                          score of the layer, so it changes no budget and no selection.     */
+} lava_layer_desc;
+
+/* Library / error plumbing ------------------------------------------------------------- */
+LAVA_API int32_t lava_version(void);            /* major*10000 + minor*100 + patch                  */
+LAVA_API const char* lava_last_error(void);     /* thread-local text of the last failure, never NULL */
+
+/* Bytes of device scratch that the score and select calls need for `n_layers` layers of this
+ * geometry processed in one call.  The first 256 bytes hold the status word; the caller
+ * should zero the workspace once after allocating it. */
+LAVA_API size_t lava_workspace_bytes(const lava_layer_desc* desc, int32_t n_layers);
+
+/* Synchronises `stream`, copies the status word to *device_status_out (host) and clears it.
+ * Returns LAVA_ERR_TIMEOUT if LAVA_DEV_WAIT_EXPIRED is set, LAVA_OK otherwise. */
+LAVA_API lava_status lava_poll_status(void* workspace, void* stream, uint32_t* device_status_out);
+
+/* C-hat of Theorem 1: the largest absolute row sum of W_O ([rows, cols], row-major, device,
+ * LAVA_F32 or LAVA_BF16) written to *c_hat_out (device float). */
+LAVA_API lava_status lava_wo_norm(const void* w_o, int32_t dtype, int64_t rows, int64_t cols,
+                         float* c_hat_out, void* stream);
+
+/* Step 1 -- LAVa score of one layer (Definition 1 with pooling and the GQA group maximum).
+ *   For each query head h (KV head g = h / G), window query t at position P+t:
+ *     A_{h,t} = softmax over keys i <= P+t of sm_scale * q_{h,t} . k_{g,i}        (Sec. 2)
+ *     a_h[i]  = (1/w) sum_t A_{h,t}[i],  i < P                                   (Definition 1)
+ *     pooled_h = pool(a_h), stride 1, centred, over the prefix only               (Sec. 5.1)
+ *     Vbar_g  = max over all n rows of the row L1 norm of V_g                     (Theorem 1)
+ *     s_g[i]  = c_hat * Vbar_g * max_{h in g} pooled_h[i]                         (Sec. 4.3)
+ *   and the layer uncertainty  e = -sum(s_hat ln s_hat) / (H_kv * n),  s_hat = s / sum(s)
+ *   over the sequence's flat score array (normalised score and entropy equations, Sec. 4.2).
+ *
+ *   q_win    [batch, H_q, w, d]  the last w queries of every sequence (post-RoPE), contiguous
+ *   k, v     per the strides in desc; v may be NULL iff vbar_in != NULL
+ *   vbar_in  [batch, H_kv] value norms supplied by the caller, or NULL to compute them from v
+ *   scores   out, float [total_scores] in the layout described at the top of this file
+ *   vbar_out out, float [batch, H_kv], may be NULL
+ *   entropy  out, double [batch]
+ * Outputs are fully overwritten; bytes beyond the stated sizes are never touched. */
+LAVA_API lava_status lava_score_layer(const lava_layer_desc* desc, const void* q_win, const void* k,
+                             const void* v, const float* vbar_in, float* scores,
+                             float* vbar_out, double* entropy, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/* The same for n_layers layers in one call.  Layer l reads q_win + l*q_layer_stride,
+ * k + l*k_layer_stride, v + l*v_layer_stride (strides in elements) and writes
+ * scores + l*total_scores, vbar_out + l*batch*H_kv, entropy + l*batch.  vbar_in, when given,
+ * is [n_layers, batch, H_kv]. */
+LAVA_API lava_status lava_score_layers(const lava_layer_desc* desc, int32_t n_layers, const void* q_win,
+                              const void* k, const void* v, int64_t q_layer_stride,
+                              int64_t k_layer_stride, int64_t v_layer_stride,
+                              const float* vbar_in, float* scores, float* vbar_out,
+                              double* entropy, void* workspace, size_t workspace_bytes,
+                              void* stream);
+
+/* Step 2 -- layer budgets (Algorithm 2: B_l = e_l / sum_l e_l * B), made integral.
+ *   entropy          double [n_layers, batch]
+ *   total_budget     int64 [batch]: model-wide budget of each sequence in KV-head rows,
+ *                    window rows included
+ *   floor_per_layer  int64 [batch]: H_kv * w      cap_per_layer  int64 [batch]: H_kv * n_b
+ *   mode             lava_budget_mode (uniform = total/L per layer, the paper's ablation)
+ *   layer_budget     out int64 [n_layers, batch], sums to total_budget[b] over layers
+ *   layer_row_offset out int64 [n_layers*batch + 1]: exclusive prefix sums of layer_budget in
+ *                    (layer, sequence) order = first row of each (layer, sequence) in the
+ *                    packed cache
+ *   status_word      device uint32 that receives LAVA_DEV_BUDGET_INFEASIBLE (may be NULL;
+ *                    normally the workspace pointer)
+ * Rule: shares proportional to e_l are rounded by largest remainder (ties to the lower layer);
+ * layers outside [floor, cap] are clamped one side at a time (the side with the larger total
+ * violation, the floor side on a tie) and the rest is re-shared among the remaining layers.
+ * n_layers <= 256, batch <= 1024. */
+LAVA_API lava_status lava_layer_budgets(int32_t n_layers, int32_t batch, const double* entropy,
+                               const int64_t* total_budget, const int64_t* floor_per_layer,
+                               const int64_t* cap_per_layer, int32_t mode,
+                               int64_t* layer_budget, int64_t* layer_row_offset,
+                               uint32_t* status_word, void* stream);
+
+/* Step 3 -- layer-wide top-k (Algorithm 1, Evict): of a sequence's H_kv*P_b prefix scores keep
+ * the  layer_budget[b] - H_kv*w  largest; equal scores are taken in ascending flat index.
+ *   scores        float [total_scores]
+ *   layer_budget  int64 [batch] (this layer's row of lava_layer_budgets' output)
+ *   keep_idx      out int32 [total_scores]: sequence b's kept prefix positions start at the
+ *                 sequence's score offset, head after head, ascending within a head; only the
+ *                 first (layer_budget[b] - H_kv*w) entries of the segment are written
+ *   head_offsets  out int32 [batch, H_kv+1]: exclusive scan of rows per head (kept prefix
+ *                 rows + w window rows); head_offsets[b][H_kv] == min(layer_budget[b], H_kv*n_b)
+ * The per-head differences of head_offsets are the dynamic head budgets. */
+LAVA_API lava_status lava_select_topk(const lava_layer_desc* desc, const float* scores,
+                             const int64_t* layer_budget, int32_t* keep_idx,
+                             int32_t* head_offsets, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/* n_layers layers in one launch: scores/keep_idx advance by total_scores per layer,
+ * layer_budget by batch, head_offsets by batch*(H_kv+1). */
+LAVA_API lava_status lava_select_topk_layers(const lava_layer_desc* desc, int32_t n_layers,
+                                    const float* scores, const int64_t* layer_budget,
+                                    int32_t* keep_idx, int32_t* head_offsets, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+
+/* Step 4 -- gather and compact (Algorithm 1: K-hat = K (.) I, V-hat = V (.) I as a gather).
+ * For sequence b and head g the rows  layer_row_offset[b] + head_offsets[b][g] ...  of k_out /
+ * v_out receive, bit for bit, the kept prefix rows in ascending position followed by the w
+ * window rows.
+ *   layer_row_offset  int64 [batch]: this layer's entries of lava_layer_budgets' output
+ *   k_out, v_out      packed caches [rows, head_dim] of the input dtype
+ * Rows outside the ranges above are not written. */
+LAVA_API lava_status lava_compact_kv(const lava_layer_desc* desc, const void* k, const void* v,
+                            const int32_t* keep_idx, const int32_t* head_offsets,
+                            const int64_t* layer_row_offset, void* k_out, void* v_out,
+                            void* stream);
+
+/* n_layers layers in one launch (k, v advance by the layer strides; keep_idx by total_scores;
+ * head_offsets by batch*(H_kv+1); layer_row_offset by batch). */
+LAVA_API lava_status lava_compact_kv_layers(const lava_layer_desc* desc, int32_t n_layers, const void* k,
+                                   const void* v, int64_t k_layer_stride, int64_t v_layer_stride,
+                                   const int32_t* keep_idx, const int32_t* head_offsets,
+                                   const int64_t* layer_row_offset, void* k_out, void* v_out,
+                                   void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAVA_H_ */

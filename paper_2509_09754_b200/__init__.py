@@ -1,0 +1,15 @@
+"""LAVa prefill-time KV-cache eviction hot path for B200 (sm_100a).
+
+Thin ctypes binding over liblava.so (hand-written CUDA).  The functions below carry the names
+of the C ABI in include/lava.h and only marshal arguments: every step runs in the library's
+kernels.  There is no CPU or PyTorch fallback; a missing library raises at first use.
+"""
+from .binding import (  # noqa: F401
+    LAVA_BF16, LAVA_F32, LAVA_POOL_AVG, LAVA_POOL_MAX, LAVA_POOL_NONE,
+    LAVA_BUDGET_DYNAMIC, LAVA_BUDGET_UNIFORM,
+    LavaError, LayerDesc, library_path, load_library,
+    lava_version, lava_last_error, lava_workspace_bytes, lava_poll_status, lava_wo_norm,
+    lava_score_layer, lava_score_layers, lava_layer_budgets,
+    lava_select_topk, lava_select_topk_layers, lava_compact_kv, lava_compact_kv_layers,
+    EvictionPlan, evict_model,
+)

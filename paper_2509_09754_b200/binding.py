@@ -1,0 +1,313 @@
+"""ctypes binding of liblava.so: argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+LAVA_F32, LAVA_BF16 = 0, 1
+LAVA_POOL_NONE, LAVA_POOL_MAX, LAVA_POOL_AVG = 0, 1, 2
+LAVA_BUDGET_DYNAMIC, LAVA_BUDGET_UNIFORM = 0, 1
+
+_STATUS_NAMES = {0: "LAVA_OK", 1: "LAVA_ERR_INVALID_ARG", 2: "LAVA_ERR_UNSUPPORTED",
+                 3: "LAVA_ERR_WORKSPACE", 4: "LAVA_ERR_CUDA", 5: "LAVA_ERR_TIMEOUT"}
+
+
+class LavaError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("%s: %s" % (_STATUS_NAMES.get(status, str(status)), message))
+        self.status = status
+
+
+class _CDesc(ctypes.Structure):
+    _fields_ = [
+        ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("window", ctypes.c_int32),
+        ("pool_kind", ctypes.c_int32), ("pool_kernel", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("batch", ctypes.c_int32),
+        ("max_seqlen", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("cu_seqlens", ctypes.c_void_p), ("total_tokens", ctypes.c_int64),
+        ("k_stride_head", ctypes.c_int64), ("k_stride_tok", ctypes.c_int64),
+        ("v_stride_head", ctypes.c_int64), ("v_stride_tok", ctypes.c_int64),
+        ("sm_scale", ctypes.c_float), ("c_hat", ctypes.c_float),
+    ]
+
+
+_LIB = None
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "liblava.so")
+
+
+def load_library():
+    """Load liblava.so; raises if it has not been built (there is no fallback path)."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(
+            "liblava.so is missing (%s): build it with `python -m paper_2509_09754_b200.build`; "
+            "this package has no CPU or PyTorch fallback" % path)
+    lib = ctypes.CDLL(path)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    dp = ctypes.POINTER(_CDesc)
+    lib.lava_version.restype = i32
+    lib.lava_last_error.restype = ctypes.c_char_p
+    lib.lava_workspace_bytes.restype = sz
+    lib.lava_workspace_bytes.argtypes = [dp, i32]
+    lib.lava_poll_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.lava_wo_norm.argtypes = [vp, i32, i64, i64, vp, vp]
+    lib.lava_score_layer.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_score_layers.argtypes = [dp, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_layer_budgets.argtypes = [i32, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp]
+    lib.lava_select_topk.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_select_topk_layers.argtypes = [dp, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_compact_kv.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.lava_compact_kv_layers.argtypes = [dp, i32, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp]
+    for name in ("lava_poll_status", "lava_wo_norm", "lava_score_layer", "lava_score_layers",
+                 "lava_layer_budgets", "lava_select_topk", "lava_select_topk_layers",
+                 "lava_compact_kv", "lava_compact_kv_layers"):
+        getattr(lib, name).restype = i32
+    _LIB = lib
+    return lib
+
+
+def _check(status: int):
+    if status != 0:
+        raise LavaError(status, load_library().lava_last_error().decode("utf-8", "replace"))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return LAVA_F32
+    if t.dtype == torch.bfloat16:
+        return LAVA_BF16
+    raise LavaError(2, "unsupported tensor dtype %s" % t.dtype)
+
+
+@dataclass
+class LayerDesc:
+    """Host-side mirror of lava_layer_desc.  K/V layout: [H_kv, total_tokens, d] views with
+    arbitrary head/token strides (last dim contiguous)."""
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    window: int
+    pool_kind: int = LAVA_POOL_MAX
+    pool_kernel: int = 7
+    dtype: int = LAVA_BF16
+    batch: int = 1
+    max_seqlen: int = 0
+    cu_seqlens: Optional[torch.Tensor] = None     # device int32 [batch + 1]
+    total_tokens: int = 0
+    k_stride_head: int = 0
+    k_stride_tok: int = 0
+    v_stride_head: int = 0
+    v_stride_tok: int = 0
+    sm_scale: float = 0.0
+    c_hat: float = 0.0
+
+    @staticmethod
+    def for_tensors(q_win: torch.Tensor, k: torch.Tensor, v: Optional[torch.Tensor], window: int,
+                    pool_kind: int = LAVA_POOL_MAX, pool_kernel: int = 7,
+                    cu_seqlens: Optional[torch.Tensor] = None, max_seqlen: int = 0,
+                    sm_scale: float = 0.0, c_hat: float = 0.0) -> "LayerDesc":
+        """q_win [batch, H_q, w, d]; k, v [H_kv, total_tokens, d] (one layer's views)."""
+        batch, hq, w, d = q_win.shape
+        hkv, total, _ = k.shape
+        vv = v if v is not None else k
+        return LayerDesc(
+            n_q_heads=hq, n_kv_heads=hkv, head_dim=d, window=window, pool_kind=pool_kind,
+            pool_kernel=pool_kernel, dtype=_dtype_code(k), batch=batch, max_seqlen=max_seqlen,
+            cu_seqlens=cu_seqlens, total_tokens=total, k_stride_head=k.stride(0),
+            k_stride_tok=k.stride(1), v_stride_head=vv.stride(0), v_stride_tok=vv.stride(1),
+            sm_scale=sm_scale, c_hat=c_hat)
+
+    @property
+    def total_scores(self) -> int:
+        return self.n_kv_heads * (self.total_tokens - self.batch * self.window)
+
+    def to_c(self) -> _CDesc:
+        return _CDesc(self.n_q_heads, self.n_kv_heads, self.head_dim, self.window, self.pool_kind,
+                      self.pool_kernel, self.dtype, self.batch, self.max_seqlen, 0,
+                      None if self.cu_seqlens is None else self.cu_seqlens.data_ptr(),
+                      self.total_tokens, self.k_stride_head, self.k_stride_tok,
+                      self.v_stride_head, self.v_stride_tok, self.sm_scale, self.c_hat)
+
+
+# ----------------------------------------------------------------------------- plumbing
+def lava_version() -> int:
+    return int(load_library().lava_version())
+
+
+def lava_last_error() -> str:
+    return load_library().lava_last_error().decode("utf-8", "replace")
+
+
+def lava_workspace_bytes(desc: LayerDesc, n_layers: int = 1) -> int:
+    c = desc.to_c()
+    n = int(load_library().lava_workspace_bytes(ctypes.byref(c), n_layers))
+    if n == 0:
+        raise LavaError(1, lava_last_error())
+    return n
+
+
+def lava_poll_status(workspace: torch.Tensor, stream=None) -> int:
+    word = ctypes.c_uint32(0)
+    _check(load_library().lava_poll_status(_ptr(workspace), _stream(stream), ctypes.byref(word)))
+    return int(word.value)
+
+
+def lava_wo_norm(w_o: torch.Tensor, c_hat_out: torch.Tensor, stream=None) -> None:
+    rows, cols = w_o.shape
+    _check(load_library().lava_wo_norm(_ptr(w_o), _dtype_code(w_o), rows, cols, _ptr(c_hat_out),
+                                       _stream(stream)))
+
+
+# ----------------------------------------------------------------------------- the four steps
+def lava_score_layer(desc: LayerDesc, q_win, k, v, vbar_in, scores, vbar_out, entropy, workspace,
+                     stream=None) -> None:
+    c = desc.to_c()
+    _check(load_library().lava_score_layer(
+        ctypes.byref(c), _ptr(q_win), _ptr(k), _ptr(v), _ptr(vbar_in), _ptr(scores),
+        _ptr(vbar_out), _ptr(entropy), _ptr(workspace), workspace.numel() * workspace.element_size(),
+        _stream(stream)))
+
+
+def lava_score_layers(desc: LayerDesc, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
+                      v_layer_stride, vbar_in, scores, vbar_out, entropy, workspace,
+                      stream=None) -> None:
+    c = desc.to_c()
+    _check(load_library().lava_score_layers(
+        ctypes.byref(c), n_layers, _ptr(q_win), _ptr(k), _ptr(v), q_layer_stride, k_layer_stride,
+        v_layer_stride, _ptr(vbar_in), _ptr(scores), _ptr(vbar_out), _ptr(entropy),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def lava_layer_budgets(n_layers, batch, entropy, total_budget, floor_per_layer, cap_per_layer,
+                       mode, layer_budget, layer_row_offset, status_word=None, stream=None) -> None:
+    _check(load_library().lava_layer_budgets(
+        n_layers, batch, _ptr(entropy), _ptr(total_budget), _ptr(floor_per_layer),
+        _ptr(cap_per_layer), mode, _ptr(layer_budget), _ptr(layer_row_offset), _ptr(status_word),
+        _stream(stream)))
+
+
+def _ws_args(workspace):
+    if workspace is None:
+        return None, 0
+    return _ptr(workspace), workspace.numel() * workspace.element_size()
+
+
+def lava_select_topk(desc: LayerDesc, scores, layer_budget, keep_idx, head_offsets,
+                     workspace=None, stream=None) -> None:
+    c = desc.to_c()
+    wp, wb = _ws_args(workspace)
+    _check(load_library().lava_select_topk(ctypes.byref(c), _ptr(scores), _ptr(layer_budget),
+                                           _ptr(keep_idx), _ptr(head_offsets), wp, wb,
+                                           _stream(stream)))
+
+
+def lava_select_topk_layers(desc: LayerDesc, n_layers, scores, layer_budget, keep_idx,
+                            head_offsets, workspace=None, stream=None) -> None:
+    c = desc.to_c()
+    wp, wb = _ws_args(workspace)
+    _check(load_library().lava_select_topk_layers(
+        ctypes.byref(c), n_layers, _ptr(scores), _ptr(layer_budget), _ptr(keep_idx),
+        _ptr(head_offsets), wp, wb, _stream(stream)))
+
+
+def lava_compact_kv(desc: LayerDesc, k, v, keep_idx, head_offsets, layer_row_offset, k_out, v_out,
+                    stream=None) -> None:
+    c = desc.to_c()
+    _check(load_library().lava_compact_kv(
+        ctypes.byref(c), _ptr(k), _ptr(v), _ptr(keep_idx), _ptr(head_offsets),
+        _ptr(layer_row_offset), _ptr(k_out), _ptr(v_out), _stream(stream)))
+
+
+def lava_compact_kv_layers(desc: LayerDesc, n_layers, k, v, k_layer_stride, v_layer_stride,
+                           keep_idx, head_offsets, layer_row_offset, k_out, v_out,
+                           stream=None) -> None:
+    c = desc.to_c()
+    _check(load_library().lava_compact_kv_layers(
+        ctypes.byref(c), n_layers, _ptr(k), _ptr(v), k_layer_stride, v_layer_stride,
+        _ptr(keep_idx), _ptr(head_offsets), _ptr(layer_row_offset), _ptr(k_out), _ptr(v_out),
+        _stream(stream)))
+
+
+# ----------------------------------------------------------------------------- whole model
+@dataclass
+class EvictionPlan:
+    """Device buffers of one full-model eviction (allocated once, reused every step)."""
+    desc: LayerDesc
+    n_layers: int
+    total_budget: torch.Tensor       # int64 [batch]
+    floor: torch.Tensor              # int64 [batch]
+    cap: torch.Tensor                # int64 [batch]
+    scores: torch.Tensor             # float [L, total_scores]
+    vbar: torch.Tensor               # float [L, batch, H_kv]
+    entropy: torch.Tensor            # double [L, batch]
+    layer_budget: torch.Tensor       # int64 [L, batch]
+    layer_row_offset: torch.Tensor   # int64 [L*batch + 1]
+    keep_idx: torch.Tensor           # int32 [L, total_scores]
+    head_offsets: torch.Tensor       # int32 [L, batch, H_kv + 1]
+    k_out: torch.Tensor              # [sum of budgets, d]
+    v_out: torch.Tensor
+    workspace: torch.Tensor          # uint8
+
+    @staticmethod
+    def create(desc: LayerDesc, n_layers: int, total_budget, seq_lens, device="cuda",
+               kv_dtype=torch.bfloat16) -> "EvictionPlan":
+        batch, hkv = desc.batch, desc.n_kv_heads
+        i64 = dict(dtype=torch.int64, device=device)
+        tb = torch.tensor([int(x) for x in total_budget], **i64)
+        floor = torch.tensor([hkv * desc.window] * batch, **i64)
+        cap = torch.tensor([hkv * int(n) for n in seq_lens], **i64)
+        rows = int(sum(int(x) for x in total_budget))
+        ts = desc.total_scores
+        ws = torch.zeros(lava_workspace_bytes(desc, n_layers), dtype=torch.uint8, device=device)
+        return EvictionPlan(
+            desc=desc, n_layers=n_layers, total_budget=tb, floor=floor, cap=cap,
+            scores=torch.empty((n_layers, ts), dtype=torch.float32, device=device),
+            vbar=torch.empty((n_layers, batch, hkv), dtype=torch.float32, device=device),
+            entropy=torch.empty((n_layers, batch), dtype=torch.float64, device=device),
+            layer_budget=torch.empty((n_layers, batch), **i64),
+            layer_row_offset=torch.empty((n_layers * batch + 1,), **i64),
+            keep_idx=torch.empty((n_layers, ts), dtype=torch.int32, device=device),
+            head_offsets=torch.empty((n_layers, batch, hkv + 1), dtype=torch.int32, device=device),
+            k_out=torch.empty((rows, desc.head_dim), dtype=kv_dtype, device=device),
+            v_out=torch.empty((rows, desc.head_dim), dtype=kv_dtype, device=device),
+            workspace=ws)
+
+
+def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC,
+                stream=None) -> None:
+    """One full-model eviction: score all layers, budgets, layer-wide top-k, compaction.
+
+    q_win [L, batch, H_q, w, d]; k, v [L, H_kv, total_tokens, d] (layer-strided views allowed).
+    Four library calls, all enqueued on the current stream; nothing is computed in Python.
+    """
+    d, nl = plan.desc, plan.n_layers
+    lava_score_layers(d, nl, q_win, k, v, q_win.stride(0), k.stride(0), v.stride(0), None,
+                      plan.scores, plan.vbar, plan.entropy, plan.workspace, stream)
+    lava_layer_budgets(nl, d.batch, plan.entropy, plan.total_budget, plan.floor, plan.cap, mode,
+                       plan.layer_budget, plan.layer_row_offset, plan.workspace, stream)
+    lava_select_topk_layers(d, nl, plan.scores, plan.layer_budget, plan.keep_idx,
+                            plan.head_offsets, plan.workspace, stream)
+    lava_compact_kv_layers(d, nl, k, v, k.stride(0), v.stride(0), plan.keep_idx,
+                           plan.head_offsets, plan.layer_row_offset, plan.k_out, plan.v_out,
+                           stream)

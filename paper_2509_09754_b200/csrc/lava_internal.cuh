@@ -1,0 +1,82 @@
+// Internal declarations shared by the translation units of liblava (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lava.h"
+
+namespace lava {
+
+// Geometry handed to kernels by value.
+struct Geom {
+  int n_q_heads, n_kv_heads, group, head_dim, window, w_pad;
+  int pool_kind, pool_kernel, pool_radius, dtype, batch, max_seqlen;
+  const int* cu_seqlens;
+  long long total_tokens, total_scores;
+  long long k_sh, k_st, v_sh, v_st;  // strides in elements
+  float scale_log2;                  // sm_scale * log2(e): logits are kept in the base-2 domain
+  float c_hat;
+};
+
+struct SeqInfo {
+  long long tok0;       // first token of the sequence in the concatenated token axis
+  int n;                // sequence length
+  int prefix;           // P = n - w (0 if the sequence is not longer than the window)
+  long long score_off;  // offset of the sequence's flat score array inside a layer
+};
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+__device__ inline SeqInfo seq_info(const Geom& g, int b) {
+  SeqInfo s;
+  if (g.cu_seqlens) {
+    s.tok0 = g.cu_seqlens[b];
+    s.n = g.cu_seqlens[b + 1] - g.cu_seqlens[b];
+  } else {
+    s.tok0 = 0;
+    s.n = (int)g.total_tokens;
+  }
+  s.prefix = s.n > g.window ? s.n - g.window : 0;
+  s.score_off = (long long)g.n_kv_heads * (s.tok0 - (long long)b * g.window);
+  return s;
+}
+
+// Workspace layout (byte offsets from the workspace base), identical for every caller.
+struct Workspace {
+  static constexpr size_t kStatusBytes = 256;
+  static constexpr int kSlice = 512;    // keys per block in the generic score kernels
+  static constexpr int kVSlice = 1024;  // V rows per block in the value-norm kernel
+  size_t off_vpart, off_stats, off_lse, off_vbar, off_ent, off_sm100, total;
+  int n_slices, n_vslices;
+};
+Workspace workspace_layout(const lava_layer_desc* d, int n_layers);
+
+// Host-side error plumbing.
+lava_status fail(lava_status st, const char* fmt, ...);
+lava_status check_cuda(cudaError_t e, const char* what);
+lava_status make_geom(const lava_layer_desc* d, Geom* out);
+
+// Launchers implemented in the kernel translation units.  Each returns LAVA_OK or the status of
+// a failed launch; all run on `stream`.
+lava_status launch_score_generic(const Geom& g, int n_layers, const void* q, const void* k,
+                                 const void* v, long long q_ls, long long k_ls, long long v_ls,
+                                 const float* vbar_in, float* scores, float* vbar_out,
+                                 double* entropy, char* ws, const Workspace& lay,
+                                 cudaStream_t stream);
+lava_status launch_wo_norm(const void* w_o, int dtype, long long rows, long long cols,
+                           float* out, cudaStream_t stream);
+lava_status launch_budgets(int n_layers, int batch, const double* entropy,
+                           const long long* total, const long long* lo, const long long* hi,
+                           int mode, long long* budget, long long* row_off, unsigned* status,
+                           cudaStream_t stream);
+lava_status launch_select(const Geom& g, int n_layers, const float* scores,
+                          const long long* layer_budget, int* keep_idx, int* head_offsets,
+                          unsigned* status, cudaStream_t stream);
+lava_status launch_compact(const Geom& g, int n_layers, const void* k, const void* v,
+                           long long k_ls, long long v_ls, const int* keep_idx,
+                           const int* head_offsets, const long long* row_off, void* k_out,
+                           void* v_out, cudaStream_t stream);
+
+}  // namespace lava

@@ -1,0 +1,88 @@
+"""Host-side checks of the C ABI: the library loads, exports every declared symbol, and
+rejects bad arguments before any launch (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2509_09754_b200 as lava
+from paper_2509_09754_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            names |= set(re.findall(r"LAVA_API[^;(]*?\b(lava_\w+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2509_09754_b200.build import build_library
+    build_library()
+    lib = lava.load_library()
+    names = _declared_symbols()
+    assert {"lava_score_layer", "lava_layer_budgets", "lava_select_topk", "lava_compact_kv"} <= names
+    for name in names:
+        assert hasattr(lib, name), name
+    assert lava.lava_version() >= 100
+
+
+def _desc(**kw):
+    base = dict(n_q_heads=4, n_kv_heads=2, head_dim=64, window=16, total_tokens=512,
+                k_stride_head=512 * 64, k_stride_tok=64, v_stride_head=512 * 64, v_stride_tok=64)
+    base.update(kw)
+    return lava.LayerDesc(**base)
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(n_q_heads=5), 1), (dict(head_dim=96), 2), (dict(window=0), 1), (dict(window=200), 2),
+    (dict(pool_kernel=4), 1), (dict(dtype=7), 1), (dict(batch=2), 1), (dict(total_tokens=8), 1),
+    (dict(k_stride_tok=60), 1), (dict(k_stride_tok=32), 1), (dict(sm_scale=-1.0), 1),
+])
+def test_bad_geometry_is_rejected_on_the_host(kw, status):
+    lib = lava.load_library()
+    c = _desc(**kw).to_c()
+    assert lib.lava_workspace_bytes(ctypes.byref(c), 1) == 0
+    rc = lib.lava_score_layer(ctypes.byref(c), 16, 16, 16, None, 16, None, 16, 16, 1 << 30, None)
+    assert rc == status
+    assert len(lava.lava_last_error()) > 0
+
+
+def test_null_misaligned_and_workspace_errors():
+    lib = lava.load_library()
+    c = _desc().to_c()
+    need = lib.lava_workspace_bytes(ctypes.byref(c), 1)
+    assert need > 256
+    assert lib.lava_score_layer(ctypes.byref(c), None, 16, 16, None, 16, None, 16, 16, need, None) == 1
+    assert lib.lava_score_layer(ctypes.byref(c), 16, 16, None, None, 16, None, 16, 16, need, None) == 1
+    assert lib.lava_score_layer(ctypes.byref(c), 16, 24, 16, None, 16, None, 16, 16, need, None) == 1
+    assert lib.lava_score_layer(ctypes.byref(c), 16, 16, 16, None, 16, None, 16, None, need, None) == 3
+    assert lib.lava_score_layer(ctypes.byref(c), 16, 16, 16, None, 16, None, 16, 16, need - 1, None) == 3
+    assert "workspace" in lava.lava_last_error()
+    assert lib.lava_layer_budgets(0, 1, 16, 16, 16, 16, 0, 16, 16, None, None) == 2
+    assert lib.lava_layer_budgets(4, 1, 16, 16, 16, 16, 9, 16, 16, None, None) == 1
+    assert lib.lava_layer_budgets(4, 1, None, 16, 16, 16, 0, 16, 16, None, None) == 1
+    assert lib.lava_select_topk(ctypes.byref(c), None, 16, 16, 16, None, 0, None) == 1
+    assert lib.lava_compact_kv(ctypes.byref(c), 16, 16, 16, 16, 16, 24, 16, None) == 1
+    assert lib.lava_compact_kv(None, 16, 16, 16, 16, 16, 16, 16, None) == 1
+    assert lib.lava_wo_norm(16, 0, 0, 4, 16, None) == 1
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "library_path", lambda: "/nonexistent/liblava.so")
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        binding.load_library()
+
+
+def test_workspace_grows_with_layers_and_context():
+    a = lava.lava_workspace_bytes(_desc(), 1)
+    b = lava.lava_workspace_bytes(_desc(), 4)
+    c = lava.lava_workspace_bytes(_desc(total_tokens=4096, k_stride_head=4096 * 64,
+                                        v_stride_head=4096 * 64), 1)
+    assert a < b and a < c
