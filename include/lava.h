@@ -197,6 +197,35 @@ LAVA_API lava_status lava_compact_kv_layers(const lava_layer_desc* desc, int32_t
                                    const int64_t* layer_row_offset, void* k_out, void* v_out,
                                    void* stream);
 
+/* Host-buffer path -- one full-model eviction (steps 1-4 over all layers) for callers whose
+ * Q window, K and V live in HOST memory (pinned memory gives asynchronous copies).
+ * Layer l is copied to the device on an internal copy stream while layer l-1 is being scored
+ * on `stream`; budgets, selection and compaction follow, and the results are copied back.
+ * Everything is asynchronous with respect to the host: the host buffers must stay valid, and
+ * the outputs are complete, once `stream` has been synchronised by the caller.
+ *   desc              geometry; desc->cu_seqlens is ignored (sequence lengths come from
+ *                     seq_lens), strides are ignored (host arrays are dense)
+ *   q_win, k, v       HOST, dense [L, batch, H_q, w, d] and [L, H_kv, total_tokens, d]
+ *   seq_lens          HOST int32 [batch]
+ *   total_budget      HOST int64 [batch]
+ *   layer_budget      HOST out int64 [L, batch]
+ *   head_offsets      HOST out int32 [L, batch, H_kv+1]
+ *   k_out, v_out      HOST out packed caches [sum(total_budget), d]
+ *   arena             DEVICE scratch of at least lava_host_arena_bytes() bytes, 256-byte
+ *                     aligned; holds the staged inputs, all intermediates and the packed cache
+ * The first call on a device creates one internal stream and a few events (host resources). */
+LAVA_API size_t lava_host_arena_bytes(const lava_layer_desc* desc, int32_t n_layers,
+                                      int64_t total_budget_rows);
+LAVA_API lava_status lava_evict_model_host(const lava_layer_desc* desc, int32_t n_layers,
+                                           const void* q_win, const void* k, const void* v,
+                                           const int32_t* seq_lens, const int64_t* total_budget,
+                                           int32_t mode, int64_t* layer_budget,
+                                           int32_t* head_offsets, void* k_out, void* v_out,
+                                           void* arena, size_t arena_bytes, void* stream);
+
+/* Number of kernel launches this library has enqueued from the calling process so far. */
+LAVA_API int64_t lava_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -69,6 +69,12 @@ def load_library():
     lib.lava_select_topk_layers.argtypes = [dp, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.lava_compact_kv.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.lava_compact_kv_layers.argtypes = [dp, i32, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp]
+    lib.lava_host_arena_bytes.restype = sz
+    lib.lava_host_arena_bytes.argtypes = [dp, i32, i64]
+    lib.lava_evict_model_host.argtypes = [dp, i32, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_evict_model_host.restype = i32
+    lib.lava_launch_count.restype = i64
+    lib.lava_launch_count.argtypes = []
     for name in ("lava_poll_status", "lava_wo_norm", "lava_score_layer", "lava_score_layers",
                  "lava_layer_budgets", "lava_select_topk", "lava_select_topk_layers",
                  "lava_compact_kv", "lava_compact_kv_layers"):
@@ -311,3 +317,28 @@ def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC
     lava_compact_kv_layers(d, nl, k, v, k.stride(0), v.stride(0), plan.keep_idx,
                            plan.head_offsets, plan.layer_row_offset, plan.k_out, plan.v_out,
                            stream)
+
+
+# ----------------------------------------------------------------------------- host buffers
+def lava_launch_count() -> int:
+    return int(load_library().lava_launch_count())
+
+
+def lava_host_arena_bytes(desc: LayerDesc, n_layers: int, total_budget_rows: int) -> int:
+    c = desc.to_c()
+    n = int(load_library().lava_host_arena_bytes(ctypes.byref(c), n_layers, total_budget_rows))
+    if n == 0:
+        raise LavaError(1, lava_last_error())
+    return n
+
+
+def lava_evict_model_host(desc: LayerDesc, n_layers, q_win, k, v, seq_lens, total_budget, mode,
+                          layer_budget, head_offsets, k_out, v_out, arena, stream=None) -> None:
+    """All tensor arguments except ``arena`` are HOST tensors (pinned for asynchronous copies);
+    seq_lens int32 [batch], total_budget int64 [batch].  Results are complete after the stream
+    has been synchronised."""
+    c = desc.to_c()
+    _check(load_library().lava_evict_model_host(
+        ctypes.byref(c), n_layers, _ptr(q_win), _ptr(k), _ptr(v), _ptr(seq_lens),
+        _ptr(total_budget), mode, _ptr(layer_budget), _ptr(head_offsets), _ptr(k_out), _ptr(v_out),
+        _ptr(arena), arena.numel() * arena.element_size(), _stream(stream)))

@@ -177,6 +177,7 @@ lava_status launch_budgets(int n_layers, int batch, const double* entropy, const
   budgets_kernel<<<batch, threads, 0, stream>>>(n_layers, batch, entropy, total, lo, hi, mode,
                                                 budget, status);
   row_offsets_kernel<<<1, 256, 0, stream>>>(n_layers * batch, budget, row_off);
+  count_launches(2);
   return check_cuda(cudaGetLastError(), "layer_budgets launch");
 }
 

@@ -60,6 +60,7 @@ lava_status launch_compact(const Geom& g, int n_layers, const void* k, const voi
   compact_kernel<<<grid, 256, 0, stream>>>(g, (const char*)k, (const char*)v, k_ls, v_ls, keep_idx,
                                            head_offsets, row_off, (char*)k_out, (char*)v_out,
                                            blocks_per_head);
+  count_launches(1);
   return check_cuda(cudaGetLastError(), "compact_kv launch");
 }
 

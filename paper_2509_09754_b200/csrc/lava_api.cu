@@ -4,11 +4,16 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "lava_internal.cuh"
 
 namespace lava {
 
 static thread_local char g_error[512] = "";
+static std::atomic<long long> g_launches{0};
+
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 lava_status fail(lava_status st, const char* fmt, ...) {
   va_list ap;
@@ -123,6 +128,8 @@ using namespace lava;
 extern "C" {
 
 int32_t lava_version(void) { return 100; }
+
+int64_t lava_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* lava_last_error(void) { return g_error; }
 

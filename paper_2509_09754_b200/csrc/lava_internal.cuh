@@ -57,6 +57,7 @@ Workspace workspace_layout(const lava_layer_desc* d, int n_layers);
 lava_status fail(lava_status st, const char* fmt, ...);
 lava_status check_cuda(cudaError_t e, const char* what);
 lava_status make_geom(const lava_layer_desc* d, Geom* out);
+void count_launches(int n);  // bookkeeping for lava_launch_count()
 
 // Launchers implemented in the kernel translation units.  Each returns LAVA_OK or the status of
 // a failed launch; all run on `stream`.

@@ -438,6 +438,7 @@ lava_status launch_score_generic(const Geom& g, int n_layers, const void* q, con
                                                          lay.n_slices);
   }
   entropy_finalize_kernel<<<problems, 32, 0, stream>>>(g, ent_part, lay.n_slices, entropy);
+  count_launches(vbar_in ? 4 : 5);
   return check_cuda(cudaGetLastError(), "score (generic) launch");
 }
 
@@ -470,6 +471,7 @@ __global__ void wo_norm_kernel(const void* w_o, int dtype, long long rows, long 
 lava_status launch_wo_norm(const void* w_o, int dtype, long long rows, long long cols, float* out,
                            cudaStream_t stream) {
   wo_norm_kernel<<<1, 1024, 0, stream>>>(w_o, dtype, rows, cols, out);
+  count_launches(1);
   return check_cuda(cudaGetLastError(), "wo_norm launch");
 }
 

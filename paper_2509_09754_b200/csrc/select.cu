@@ -201,6 +201,7 @@ lava_status launch_select(const Geom& g, int n_layers, const float* scores,
   dim3 grid(kCluster, n_layers * g.batch);
   select_topk_kernel<<<grid, kThreads, 0, stream>>>(g, scores, layer_budget, keep_idx,
                                                     head_offsets);
+  count_launches(1);
   return check_cuda(cudaGetLastError(), "select_topk launch");
 }
 

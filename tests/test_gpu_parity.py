@@ -184,3 +184,29 @@ def test_wo_norm():
     out = torch.zeros(1, device="cuda")
     lava.lava_wo_norm(w_o, out)
     assert abs(float(out) - O.wo_norm(w_o.cpu().numpy())) < 1e-4 * float(out)
+
+
+def test_host_buffer_path_equals_device_path():
+    cfg = get_config("mistral7b_ragged").scaled(seq_lens=(640, 901), n_layers=3, budget_per_head=96)
+    q, k, v, cu = upload_model(cfg)
+    plan = make_plan(cfg, q, k, v, cu)
+    lava.evict_model(plan, q, k, v)
+    rows = plan.k_out.shape[0]
+    L, hkv = cfg.n_layers, cfg.n_kv_heads
+    pin = lambda x: x.cpu().pin_memory()
+    out_budget = torch.empty((L, cfg.batch), dtype=torch.int64).pin_memory()
+    out_hoff = torch.empty((L, cfg.batch, hkv + 1), dtype=torch.int32).pin_memory()
+    out_k = torch.empty((rows, cfg.head_dim), dtype=k.dtype).pin_memory()
+    out_v = torch.empty((rows, cfg.head_dim), dtype=k.dtype).pin_memory()
+    budgets = [cfg.total_budget(b) for b in range(cfg.batch)]
+    arena = torch.empty(lava.lava_host_arena_bytes(plan.desc, L, rows), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        lava.lava_evict_model_host(plan.desc, L, pin(q), pin(k), pin(v),
+                                   torch.tensor(cfg.seq_lens, dtype=torch.int32),
+                                   torch.tensor(budgets, dtype=torch.int64), 0, out_budget, out_hoff,
+                                   out_k, out_v, arena)
+        torch.cuda.synchronize()
+        assert torch.equal(out_budget, plan.layer_budget.cpu())
+        assert torch.equal(out_hoff, plan.head_offsets.cpu())
+        assert torch.equal(out_k.view(torch.int16), plan.k_out.cpu().view(torch.int16))
+        assert torch.equal(out_v.view(torch.int16), plan.v_out.cpu().view(torch.int16))
