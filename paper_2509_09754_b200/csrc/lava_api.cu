@@ -2,6 +2,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <atomic>
@@ -117,6 +118,8 @@ Workspace workspace_layout(const lava_layer_desc* d, int n_layers) {
   w.off_ent = off;
   off = round_up(off + problems * d->n_kv_heads * w.n_slices * sizeof(double2), 256);
   w.off_sm100 = off;
+  Geom g;
+  if (make_geom(d, &g) == LAVA_OK && sm100_supported(g)) off += sm100_layout(g, n_layers).total;
   w.total = off;
   return w;
 }
@@ -187,6 +190,11 @@ lava_status lava_score_layers(const lava_layer_desc* desc, int32_t n_layers, con
     return fail(LAVA_ERR_WORKSPACE, "workspace too small: %zu < %zu bytes", workspace_bytes,
                 lay.total);
   if (!aligned16(workspace)) return fail(LAVA_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
+  const char* force = getenv("LAVA_FORCE_GENERIC");
+  if (sm100_supported(g) && !(force && force[0] == '1'))
+    return launch_score_sm100(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
+                              v_layer_stride, vbar_in, scores, vbar_out, entropy,
+                              (char*)workspace, lay.off_sm100, (cudaStream_t)stream);
   return launch_score_generic(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
                               v_layer_stride, vbar_in, scores, vbar_out, entropy,
                               (char*)workspace, lay, (cudaStream_t)stream);

@@ -66,6 +66,17 @@ lava_status launch_score_generic(const Geom& g, int n_layers, const void* q, con
                                  const float* vbar_in, float* scores, float* vbar_out,
                                  double* entropy, char* ws, const Workspace& lay,
                                  cudaStream_t stream);
+// Blackwell tensor-core score path (bf16, head_dim 128, G*w <= 128).
+struct Sm100Layout {
+  int heads_total, tiles1, tiles2, out_keys;
+  size_t off_sync, sync_bytes, off_part, off_lse, off_ent, total;
+};
+bool sm100_supported(const Geom& g);
+Sm100Layout sm100_layout(const Geom& g, int n_layers);
+lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const void* k,
+                               const void* v, long long q_ls, long long k_ls, long long v_ls,
+                               const float* vbar_in, float* scores, float* vbar_out,
+                               double* entropy, char* ws_base, size_t ws_off, cudaStream_t stream);
 lava_status launch_wo_norm(const void* w_o, int dtype, long long rows, long long cols,
                            float* out, cudaStream_t stream);
 lava_status launch_budgets(int n_layers, int batch, const double* entropy,
