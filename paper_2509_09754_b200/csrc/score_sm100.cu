@@ -1,25 +1,28 @@
 // LAVa score, Blackwell path: bf16, head_dim 128, G*w <= 128, w in {16, 32, 64, 128}.
 //
-// One persistent, warp-specialised kernel (one CTA per SM) runs two pipelines over 128-key
-// tiles of K, both fed by TMA into 128B-swizzled shared memory and contracted with tcgen05.mma
-// into TMEM:
+// One persistent, warp-specialised kernel (one CTA per SM, cooperative launch so that every CTA
+// is resident) runs two pipelines over 128-key tiles of K, both fed by TMA into 128B-swizzled
+// shared memory and contracted with tcgen05.mma into TMEM:
 //
 //   pass 1 (statistics)  S = Q_g K^T  (rows = the group's G*w window queries, columns = keys)
-//       one thread per row reads its TMEM lane: masked row max and sum of exp2 over the keys
-//       the query may see (Sec. 2: softmax over i <= j), published per (head, tile); four more
-//       warps stream the matching V rows for the value norm (Theorem 1: max_k ||V[k]||_1).
-//       The CTA that publishes the last tile of a head folds the partials into one
-//       log-sum-exp per query and raises the head's ready flag.
+//       one thread per row reads its TMEM lane and keeps a running (max, sum of exp2) over the
+//       keys the query may see (Sec. 2: softmax over i <= j).  Work is dealt to CTAs in chunks
+//       of a few consecutive tiles of one head; a chunk's statistics leave the CTA once, through
+//       a publisher warp.  The publisher that completes a head folds the chunk partials, in
+//       chunk order, into one log-sum-exp per query and raises the head's ready flag.  Four more
+//       warps stream the chunk's V rows for the value norm (Theorem 1: max_k ||V[k]||_1).
 //   pass 2 (scores)      S^T = K Q_g^T (rows = keys, columns = window queries)
 //       one thread per key: a_h[i] = (1/w) sum_t exp2(z - lse_t) per query head in registers,
 //       pooled over the token axis through shared memory, scaled by Vbar * c_hat, reduced with
-//       the GQA group maximum, written once; per-tile entropy sums go to ordered slots
+//       the GQA group maximum, written once; entropy sums go to ordered per-chunk slots
 //       (Definition 1, Sec. 4.2, Sec. 4.3, Sec. 5.1 pooling).
 //
-// K is read from HBM once: pass 2 trails pass 1 by a bounded number of heads, so its tiles are
-// still in L2.  Every wait (mbarrier, ready flag) is bounded; on expiry the kernel sets
-// LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
+// K is read from HBM once: pass 2 trails pass 1 by a bounded number of keys, so its tiles are
+// still in L2 (K tiles are loaded with an evict-last hint in pass 1 and evict-first in pass 2,
+// V rows with evict-first).  Every wait (mbarrier, ready flag, throttle) is bounded; on expiry
+// the kernel sets LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "lava_internal.cuh"
 
@@ -29,6 +32,7 @@ namespace {
 constexpr int kTile = 128;           // keys per tile
 constexpr int kThreads = 512;        // 16 warps
 constexpr int kStages = 2;           // K stages per pipeline
+constexpr int kMaxBatch = 512;       // sequences the in-kernel chunk schedule can index
 constexpr uint32_t kTileBytes = 128 * 128 * 2;  // one [128 x 128] bf16 tile = 2 swizzled blocks
 constexpr uint32_t kHalfBytes = kTileBytes / 2;
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -39,45 +43,53 @@ constexpr uint32_t kOffQ2 = kOffQ1 + kTileBytes;
 constexpr uint32_t kOffK1 = kOffQ2 + kTileBytes;
 constexpr uint32_t kOffK2 = kOffK1 + kStages * kTileBytes;
 constexpr uint32_t kOffMisc = kOffK2 + kStages * kTileBytes;  // 192 KB
-constexpr uint32_t kMiscBytes = 12288;
+constexpr uint32_t kMiscBytes = 20480;
 constexpr uint32_t kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + alignment slack
+
+struct Prep {                 // what the score warps need to know about a head
+  alignas(16) float lse[128]; // -(log2-sum-exp) per window query
+  float scale;                // Vbar * c_hat
+  float pad[3];
+};
 
 struct Misc {
   unsigned long long k1_full[kStages], k1_empty[kStages], k2_full[kStages], k2_empty[kStages];
   unsigned long long q1_full, q1_empty, q2_full, q2_empty;
   unsigned long long s1_full[2], s1_empty[2], s2_full[2], s2_empty[2];
+  unsigned long long pub_full[2], pub_empty[2], prep_full[2], prep_empty[2];
   unsigned long long drain;
+  volatile long long p2_pos;  // first key (global key coordinate) pass 2 has not finished yet
   uint32_t tmem_base;
   volatile int abort_flag;
-  volatile int p2_head;     // head (linear index) the score warps are working on
-  int last_flag;
-  alignas(16) float lse[128];  // -(log2-sum-exp) of the current pass-2 head, per window query
-  alignas(16) float a[2][8][kTile];  // window-mean attention per (query head, key) of the current tile
+  int sched_total1, sched_total2;     // chunks per layer of pass 1 / pass 2
+  alignas(16) float2 pub[2][128];     // (max, sum) of a finished pass-1 chunk, per window query
+  Prep prep[2];
+  alignas(16) float a[2][8][kTile];   // window-mean attention per (query head, key) of a tile
   float red[2][4];
-  float vmax[4];
+  int pref1[kMaxBatch + 1], pref2[kMaxBatch + 1];  // exclusive scans of chunks per sequence
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
 
 struct Sm100Params {
   Geom g;
   int n_layers;
-  int heads_total;          // n_layers * batch * H_kv
-  int tiles1_per_head;      // ceil(max_seqlen / 128)
-  int tiles2_per_head;      // ceil(max_prefix / out_keys)
+  int chunk_tiles;          // tiles per chunk
   int out_keys;             // keys a pass-2 tile owns: 128 - 2 * pool_radius
-  int lag_heads;            // pass 1 may run this many heads ahead of pass 2
+  int cph1_max, cph2_max;   // chunks per head at max_seqlen (strides of the scratch arrays)
+  long long lag_keys;       // pass 1 may run this many keys ahead of pass 2
   const float* vbar_in;
   float* scores;
   float* vbar_out;
   const char* v;
   long long v_ls;
   // scratch
-  float2* part;             // [heads_total][tiles1_per_head][128]
-  int* counters;            // [heads_total]
+  float2* part;             // [heads_total][cph1_max][128]
+  int* counters;            // [heads_total] published pass-1 chunks
   int* ready;               // [heads_total]
+  int* vcount;              // [heads_total] finished value-norm warps
   unsigned* vbar_bits;      // [heads_total]
   float* neg_lse;           // [heads_total][128]
-  double2* ent_part;        // [heads_total][tiles2_per_head]
+  double2* ent_part;        // [heads_total][cph2_max]
   unsigned* status;
 };
 
@@ -106,6 +118,16 @@ __device__ inline bool mbar_test(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ inline uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ inline uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
                                    uint32_t bar) {
   asm volatile(
@@ -115,11 +137,11 @@ __device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0,
       : "memory");
 }
 __device__ inline void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
-                                   int c3, uint32_t bar) {
+                                   int c3, uint32_t bar, uint64_t policy) {
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      ".L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
       : "memory");
 }
 __device__ inline void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
@@ -151,8 +173,9 @@ __device__ inline void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_de
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ inline void tmem_ld32(uint32_t taddr, float* v) {
+// 32 consecutive fp32 columns of this thread's TMEM lane: issue, and (separately) wait.  The
+// wait names the destination registers so that no use of them can be scheduled before it.
+__device__ inline void tmem_ld32_issue(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -165,7 +188,18 @@ __device__ inline void tmem_ld32(uint32_t taddr, float* v) {
         "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ inline void tmem_ld_wait(float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
+        "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]),
+        "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]),
+        "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
+        "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :
+      : "memory");
 }
 __device__ inline void named_barrier(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -195,6 +229,13 @@ __device__ inline int ld_acquire(const int* p) {
 __device__ inline void st_release(int* p, int v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ inline uint4 ld_stream16(const void* p, uint64_t policy) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p), "l"(policy));
+  return r;
+}
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 B apart.
 __device__ inline uint64_t make_desc(uint32_t saddr) {
@@ -209,44 +250,69 @@ __device__ inline uint64_t make_desc(uint32_t saddr) {
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
+__device__ inline void give_up(Misc* m, unsigned* status) {
+  m->abort_flag = 1;
+  atomicOr(status, LAVA_DEV_WAIT_EXPIRED);
+}
+
 // Bounded mbarrier wait.  Returns false once the CTA is aborting (unless heed_abort is false:
 // the drain waits at exit must outlast an abort to let copies in flight land).
 __device__ inline bool wait_bar(uint32_t bar, uint32_t parity, Misc* m, unsigned* status,
                                 bool heed_abort = true) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_test(bar, parity)) return true;
-    if (it > 128) {
+    if (it > 64) {
       if (heed_abort && m->abort_flag) return false;
-      __nanosleep(64);
+      __nanosleep(32);
     }
   }
-  m->abort_flag = 1;
-  atomicOr(status, LAVA_DEV_WAIT_EXPIRED);
+  give_up(m, status);
   return false;
 }
 
 // ------------------------------------------------------------------------------------------
-// item decoding (identical in every role, so no descriptors travel between warps)
+// chunk schedule (identical in every role and every CTA, so no descriptors travel)
 // ------------------------------------------------------------------------------------------
-struct Item {
+struct Chunk {
   int head;    // linear head index = (layer * batch + b) * H_kv + kvh
-  int layer, b, kvh, tile;
+  int layer, b, kvh;
+  int index;   // chunk number inside the head
+  int cph;     // chunks of this head
+  int tile0, ntiles;
   SeqInfo s;
-  bool valid;
 };
 
-__device__ inline Item decode(const Sm100Params& p, long long idx, int tiles_per_head, int pass) {
-  Item it;
-  it.head = (int)(idx / tiles_per_head);
-  it.tile = (int)(idx - (long long)it.head * tiles_per_head);
-  const int prob = it.head / p.g.n_kv_heads;
-  it.kvh = it.head - prob * p.g.n_kv_heads;
-  it.layer = prob / p.g.batch;
-  it.b = prob - it.layer * p.g.batch;
-  it.s = seq_info(p.g, it.b);
-  if (pass == 1) it.valid = (long long)it.tile * kTile < it.s.n;
-  else it.valid = (long long)it.tile * p.out_keys < it.s.prefix;
-  return it;
+__device__ inline int tiles_of(const Sm100Params& p, const SeqInfo& s, int pass) {
+  return pass == 1 ? ceil_div(s.n, kTile) : ceil_div(s.prefix, p.out_keys);
+}
+
+__device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, long long c, int pass) {
+  const int* pref = pass == 1 ? m->pref1 : m->pref2;
+  const int per_layer = pass == 1 ? m->sched_total1 : m->sched_total2;
+  Chunk ck;
+  ck.layer = (int)(c / per_layer);
+  const int r = (int)(c - (long long)ck.layer * per_layer);
+  const int hkv = p.g.n_kv_heads;
+  int lo = 0, hi = p.g.batch;  // largest b with hkv * pref[b] <= r
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (hkv * pref[mid] <= r) lo = mid; else hi = mid;
+  }
+  ck.b = lo;
+  ck.cph = pref[lo + 1] - pref[lo];
+  const int r2 = r - hkv * pref[lo];
+  ck.kvh = r2 / ck.cph;
+  ck.index = r2 - ck.kvh * ck.cph;
+  ck.head = (ck.layer * p.g.batch + ck.b) * hkv + ck.kvh;
+  ck.s = seq_info(p.g, ck.b);
+  ck.tile0 = ck.index * p.chunk_tiles;
+  ck.ntiles = min(p.chunk_tiles, tiles_of(p, ck.s, pass) - ck.tile0);
+  return ck;
+}
+
+// global key coordinate used by the pass-1 throttle
+__device__ inline long long key_pos(const Sm100Params& p, int head, long long key) {
+  return (long long)head * p.g.max_seqlen + key;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -263,8 +329,49 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Geom& g = p.g;
   const int rows_valid = g.group * W;
-  const long long items1 = (long long)p.heads_total * p.tiles1_per_head;
-  const long long items2 = (long long)p.heads_total * p.tiles2_per_head;
+
+  // ---- chunk schedule: exclusive scans of chunks per sequence, both passes -------------------
+  {
+    __shared__ int wsum[2][kThreads / 32];
+    int c1 = 0, c2 = 0;
+    if ((int)threadIdx.x < g.batch) {
+      const SeqInfo s = seq_info(g, threadIdx.x);
+      c1 = ceil_div(ceil_div(s.n, kTile), p.chunk_tiles);
+      c2 = ceil_div(ceil_div(s.prefix, p.out_keys), p.chunk_tiles);
+    }
+    int i1 = c1, i2 = c2;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y1 = __shfl_up_sync(0xffffffffu, i1, o), y2 = __shfl_up_sync(0xffffffffu, i2, o);
+      if (lane >= o) {
+        i1 += y1;
+        i2 += y2;
+      }
+    }
+    if (lane == 31) {
+      wsum[0][warp] = i1;
+      wsum[1][warp] = i2;
+    }
+    __syncthreads();
+    int b1 = 0, b2 = 0;
+    for (int wdx = 0; wdx < warp; ++wdx) {
+      b1 += wsum[0][wdx];
+      b2 += wsum[1][wdx];
+    }
+    if ((int)threadIdx.x < g.batch) {
+      m->pref1[threadIdx.x + 1] = b1 + i1;
+      m->pref2[threadIdx.x + 1] = b2 + i2;
+    }
+    if (threadIdx.x == 0) {
+      m->pref1[0] = 0;
+      m->pref2[0] = 0;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      m->sched_total1 = g.n_kv_heads * m->pref1[g.batch];
+      m->sched_total2 = g.n_kv_heads * m->pref2[g.batch];
+    }
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -282,11 +389,14 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       mbar_init(smem_u32(&m->s1_empty[s]), 128);
       mbar_init(smem_u32(&m->s2_full[s]), 1);
       mbar_init(smem_u32(&m->s2_empty[s]), 128);
+      mbar_init(smem_u32(&m->pub_full[s]), 128);
+      mbar_init(smem_u32(&m->pub_empty[s]), 1);
+      mbar_init(smem_u32(&m->prep_full[s]), 1);
+      mbar_init(smem_u32(&m->prep_empty[s]), 1);
     }
     mbar_init(smem_u32(&m->drain), 1);
     m->abort_flag = 0;
-    m->p2_head = 0;
-    m->last_flag = 0;
+    m->p2_pos = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -295,49 +405,50 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = m->tmem_base;
+  const long long total1 = (long long)p.n_layers * m->sched_total1;
+  const long long total2 = (long long)p.n_layers * m->sched_total2;
 
   if (warp == 0) {
     // ================= pass-1 producer: Q of the head, K tiles =============================
     if (lane == 0) {
-      int prev_head = -1, q_loads = 0;
-      long long n = 0;  // loads issued
-      for (long long idx = blockIdx.x; idx < items1; idx += gridDim.x) {
-        const Item it = decode(p, idx, p.tiles1_per_head, 1);
-        if (!it.valid) continue;
-        // stay within lag_heads of the score warps so pass 2 still finds its tiles in L2
+      const uint64_t keep = policy_evict_last();
+      int q_loads = 0;
+      long long n = 0;  // K loads issued
+      for (long long c = blockIdx.x; c < total1 && !m->abort_flag; c += gridDim.x) {
+        const Chunk ck = decode_chunk(p, m, c, 1);
+        // stay within lag_keys of the score warps so pass 2 still finds its tiles in L2
         {
+          const long long pos = key_pos(p, ck.head, (long long)ck.tile0 * kTile);
           uint32_t spins = 0;
-          while (it.head > m->p2_head + p.lag_heads) {
-            if (m->abort_flag) break;
+          while (pos > m->p2_pos + p.lag_keys && !m->abort_flag) {
             __nanosleep(128);
-            if (++spins > kSpinLimit) {
-              m->abort_flag = 1;
-              atomicOr(p.status, LAVA_DEV_WAIT_EXPIRED);
-              break;
-            }
+            if (++spins > kSpinLimit) give_up(m, p.status);
           }
           if (m->abort_flag) break;
         }
-        if (it.head != prev_head) {
-          if (!wait_bar(smem_u32(&m->q1_empty), (q_loads & 1) ^ 1, m, p.status)) break;
+        if (!wait_bar(smem_u32(&m->q1_empty), (q_loads & 1) ^ 1, m, p.status)) break;
+        {
           const uint32_t bar = smem_u32(&m->q1_full);
           mbar_expect_tx(bar, kTileBytes);
-          const int row0 = (it.b * g.n_q_heads + it.kvh * g.group) * W;
-          tma_load_3d(base + kOffQ1, &map_q, 0, row0, it.layer, bar);
-          tma_load_3d(base + kOffQ1 + kHalfBytes, &map_q, 64, row0, it.layer, bar);
-          prev_head = it.head;
+          const int row0 = (ck.b * g.n_q_heads + ck.kvh * g.group) * W;
+          tma_load_3d(base + kOffQ1, &map_q, 0, row0, ck.layer, bar);
+          tma_load_3d(base + kOffQ1 + kHalfBytes, &map_q, 64, row0, ck.layer, bar);
           ++q_loads;
         }
-        const int st = (int)(n % kStages);
-        if (!wait_bar(smem_u32(&m->k1_empty[st]), (uint32_t)((n / kStages) & 1) ^ 1, m, p.status))
-          break;
-        const uint32_t bar = smem_u32(&m->k1_full[st]);
-        mbar_expect_tx(bar, kTileBytes);
-        const int tok = (int)it.s.tok0 + it.tile * kTile;
-        tma_load_4d(base + kOffK1 + st * kTileBytes, &map_k, 0, tok, it.kvh, it.layer, bar);
-        tma_load_4d(base + kOffK1 + st * kTileBytes + kHalfBytes, &map_k, 64, tok, it.kvh, it.layer,
-                    bar);
-        ++n;
+        bool ok = true;
+        for (int t = 0; t < ck.ntiles && ok; ++t) {
+          const int st = (int)(n % kStages);
+          ok = wait_bar(smem_u32(&m->k1_empty[st]), (uint32_t)((n / kStages) & 1) ^ 1, m, p.status);
+          if (!ok) break;
+          const uint32_t bar = smem_u32(&m->k1_full[st]);
+          mbar_expect_tx(bar, kTileBytes);
+          const int tok = (int)ck.s.tok0 + (ck.tile0 + t) * kTile;
+          tma_load_4d(base + kOffK1 + st * kTileBytes, &map_k, 0, tok, ck.kvh, ck.layer, bar, keep);
+          tma_load_4d(base + kOffK1 + st * kTileBytes + kHalfBytes, &map_k, 64, tok, ck.kvh,
+                      ck.layer, bar, keep);
+          ++n;
+        }
+        if (!ok) break;
       }
       // copies still in flight land before this CTA gives up its shared memory
       for (long long j = (n > kStages ? n - kStages : 0); j < n; ++j)
@@ -347,37 +458,69 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         wait_bar(smem_u32(&m->q1_full), (uint32_t)((q_loads - 1) & 1), m, p.status, false);
     }
   } else if (warp == 1) {
-    // ================= pass-2 producer ======================================================
-    if (lane == 0) {
-      int prev_head = -1, q_loads = 0;
-      long long n = 0;
-      for (long long idx = blockIdx.x; idx < items2; idx += gridDim.x) {
-        const Item it = decode(p, idx, p.tiles2_per_head, 2);
-        if (!it.valid) continue;
-        if (it.head != prev_head) {
-          if (!wait_bar(smem_u32(&m->q2_empty), (q_loads & 1) ^ 1, m, p.status)) break;
+    // ================= pass-2 producer: head data for the score warps, Q, K tiles ============
+    const uint64_t drop = policy_evict_first();
+    int q_loads = 0;
+    long long n = 0, j = 0;  // K loads issued, chunks prepared
+    for (long long c = blockIdx.x; c < total2; c += gridDim.x, ++j) {
+      const Chunk ck = decode_chunk(p, m, c, 2);
+      const int slot = (int)(j & 1);
+      // wait until the head's log-sum-exp and value norm are final
+      bool ok = true;
+      if (lane == 0) {
+        const int want_v = p.vbar_in ? 0 : 4 * ceil_div(ceil_div(ck.s.n, kTile), p.chunk_tiles);
+        uint32_t spins = 0;
+        while (ld_acquire(&p.ready[ck.head]) == 0 ||
+               (want_v && ld_acquire(&p.vcount[ck.head]) < want_v)) {
+          if (m->abort_flag) break;
+          __nanosleep(64);
+          if (++spins > kSpinLimit) give_up(m, p.status);
+        }
+        ok = !m->abort_flag &&
+             wait_bar(smem_u32(&m->prep_empty[slot]), (uint32_t)((j >> 1) & 1) ^ 1, m, p.status);
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        m->prep[slot].lse[lane + 32 * q] = __ldcg(p.neg_lse + (size_t)ck.head * 128 + lane + 32 * q);
+      if (lane == 0) {
+        const float vb = p.vbar_in ? p.vbar_in[ck.head]
+                                   : __uint_as_float(__ldcg(p.vbar_bits + ck.head));
+        m->prep[slot].scale = vb * g.c_hat;
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(smem_u32(&m->prep_full[slot]));
+        ok = wait_bar(smem_u32(&m->q2_empty), (q_loads & 1) ^ 1, m, p.status);
+        if (ok) {
           const uint32_t bar = smem_u32(&m->q2_full);
           mbar_expect_tx(bar, kTileBytes);
-          const int row0 = (it.b * g.n_q_heads + it.kvh * g.group) * W;
-          tma_load_3d(base + kOffQ2, &map_q, 0, row0, it.layer, bar);
-          tma_load_3d(base + kOffQ2 + kHalfBytes, &map_q, 64, row0, it.layer, bar);
-          prev_head = it.head;
+          const int row0 = (ck.b * g.n_q_heads + ck.kvh * g.group) * W;
+          tma_load_3d(base + kOffQ2, &map_q, 0, row0, ck.layer, bar);
+          tma_load_3d(base + kOffQ2 + kHalfBytes, &map_q, 64, row0, ck.layer, bar);
           ++q_loads;
         }
-        const int st = (int)(n % kStages);
-        if (!wait_bar(smem_u32(&m->k2_empty[st]), (uint32_t)((n / kStages) & 1) ^ 1, m, p.status))
-          break;
-        const uint32_t bar = smem_u32(&m->k2_full[st]);
-        mbar_expect_tx(bar, kTileBytes);
-        // the tile starts pool_radius keys before the first key it owns (halo for pooling)
-        const int tok = (int)it.s.tok0 + it.tile * p.out_keys - g.pool_radius;
-        tma_load_4d(base + kOffK2 + st * kTileBytes, &map_k, 0, tok, it.kvh, it.layer, bar);
-        tma_load_4d(base + kOffK2 + st * kTileBytes + kHalfBytes, &map_k, 64, tok, it.kvh, it.layer,
-                    bar);
-        ++n;
+        for (int t = 0; t < ck.ntiles && ok; ++t) {
+          const int st = (int)(n % kStages);
+          ok = wait_bar(smem_u32(&m->k2_empty[st]), (uint32_t)((n / kStages) & 1) ^ 1, m, p.status);
+          if (!ok) break;
+          const uint32_t bar = smem_u32(&m->k2_full[st]);
+          mbar_expect_tx(bar, kTileBytes);
+          // the tile starts pool_radius keys before the first key it owns (halo for pooling)
+          const int tok = (int)ck.s.tok0 + (ck.tile0 + t) * p.out_keys - g.pool_radius;
+          tma_load_4d(base + kOffK2 + st * kTileBytes, &map_k, 0, tok, ck.kvh, ck.layer, bar, drop);
+          tma_load_4d(base + kOffK2 + st * kTileBytes + kHalfBytes, &map_k, 64, tok, ck.kvh,
+                      ck.layer, bar, drop);
+          ++n;
+        }
       }
-      for (long long j = (n > kStages ? n - kStages : 0); j < n; ++j)
-        wait_bar(smem_u32(&m->k2_full[j % kStages]), (uint32_t)((j / kStages) & 1), m, p.status,
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+    }
+    if (lane == 0) {
+      for (long long i = (n > kStages ? n - kStages : 0); i < n; ++i)
+        wait_bar(smem_u32(&m->k2_full[i % kStages]), (uint32_t)((i / kStages) & 1), m, p.status,
                  false);
       if (q_loads > 0)
         wait_bar(smem_u32(&m->q2_full), (uint32_t)((q_loads - 1) & 1), m, p.status, false);
@@ -385,26 +528,21 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
   } else if (warp == 2) {
     // ================= MMA issuer: serves both pipelines by polling =========================
     if (lane == 0) {
-      long long idx1 = blockIdx.x, idx2 = blockIdx.x;
+      long long c1 = blockIdx.x, c2 = blockIdx.x;
       long long n1 = 0, n2 = 0;
-      int prev1 = -1, prev2 = -1, q1_uses = 0, q2_uses = 0;
+      int t1 = 0, t2 = 0, nt1 = 0, nt2 = 0, q1_uses = 0, q2_uses = 0;
+      if (c1 < total1) nt1 = decode_chunk(p, m, c1, 1).ntiles;
+      if (c2 < total2) nt2 = decode_chunk(p, m, c2, 2).ntiles;
       uint32_t idle = 0;
-      // skip leading empty items
-      while (idx1 < items1 && !decode(p, idx1, p.tiles1_per_head, 1).valid) idx1 += gridDim.x;
-      while (idx2 < items2 && !decode(p, idx2, p.tiles2_per_head, 2).valid) idx2 += gridDim.x;
-      while (idx1 < items1 || idx2 < items2) {
+      while (c1 < total1 || c2 < total2) {
         bool progressed = false;
-        if (idx1 < items1) {
-          const Item it = decode(p, idx1, p.tiles1_per_head, 1);
+        if (c1 < total1) {
           const int st = (int)(n1 % kStages), buf = (int)(n1 & 1);
-          const bool need_q = it.head != prev1;
+          const bool need_q = t1 == 0;
           if (mbar_test(smem_u32(&m->k1_full[st]), (uint32_t)((n1 / kStages) & 1)) &&
               mbar_test(smem_u32(&m->s1_empty[buf]), (uint32_t)((n1 >> 1) & 1) ^ 1) &&
               (!need_q || mbar_test(smem_u32(&m->q1_full), (uint32_t)(q1_uses & 1)))) {
-            if (need_q) {
-              prev1 = it.head;
-              ++q1_uses;
-            }
+            if (need_q) ++q1_uses;
             tc_fence_after();
             const uint32_t d = tmem + (uint32_t)buf * 128u;
 #pragma unroll
@@ -416,25 +554,23 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
             umma_commit(smem_u32(&m->k1_empty[st]));
             umma_commit(smem_u32(&m->s1_full[buf]));
             ++n1;
-            idx1 += gridDim.x;
-            while (idx1 < items1 && !decode(p, idx1, p.tiles1_per_head, 1).valid) idx1 += gridDim.x;
-            // the query tile may be replaced once the MMAs of its last user have completed
-            if (idx1 >= items1 || decode(p, idx1, p.tiles1_per_head, 1).head != prev1)
+            if (++t1 == nt1) {
+              // the query tile may be replaced once the MMAs of its last user have completed
               umma_commit(smem_u32(&m->q1_empty));
+              t1 = 0;
+              c1 += gridDim.x;
+              if (c1 < total1) nt1 = decode_chunk(p, m, c1, 1).ntiles;
+            }
             progressed = true;
           }
         }
-        if (idx2 < items2) {
-          const Item it = decode(p, idx2, p.tiles2_per_head, 2);
+        if (c2 < total2) {
           const int st = (int)(n2 % kStages), buf = (int)(n2 & 1);
-          const bool need_q = it.head != prev2;
+          const bool need_q = t2 == 0;
           if (mbar_test(smem_u32(&m->k2_full[st]), (uint32_t)((n2 / kStages) & 1)) &&
               mbar_test(smem_u32(&m->s2_empty[buf]), (uint32_t)((n2 >> 1) & 1) ^ 1) &&
               (!need_q || mbar_test(smem_u32(&m->q2_full), (uint32_t)(q2_uses & 1)))) {
-            if (need_q) {
-              prev2 = it.head;
-              ++q2_uses;
-            }
+            if (need_q) ++q2_uses;
             tc_fence_after();
             const uint32_t d = tmem + 256u + (uint32_t)buf * 128u;
 #pragma unroll
@@ -446,24 +582,23 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
             umma_commit(smem_u32(&m->k2_empty[st]));
             umma_commit(smem_u32(&m->s2_full[buf]));
             ++n2;
-            idx2 += gridDim.x;
-            while (idx2 < items2 && !decode(p, idx2, p.tiles2_per_head, 2).valid) idx2 += gridDim.x;
-            if (idx2 >= items2 || decode(p, idx2, p.tiles2_per_head, 2).head != prev2)
+            if (++t2 == nt2) {
               umma_commit(smem_u32(&m->q2_empty));
+              t2 = 0;
+              c2 += gridDim.x;
+              if (c2 < total2) nt2 = decode_chunk(p, m, c2, 2).ntiles;
+            }
             progressed = true;
           }
         }
         if (progressed) {
           idle = 0;
-        } else {
-          if (++idle > 256) {
-            if (m->abort_flag) break;
-            __nanosleep(32);
-            if (idle > kSpinLimit) {
-              m->abort_flag = 1;
-              atomicOr(p.status, LAVA_DEV_WAIT_EXPIRED);
-              break;
-            }
+        } else if (++idle > 64) {
+          if (m->abort_flag) break;
+          __nanosleep(32);
+          if (idle > kSpinLimit) {
+            give_up(m, p.status);
+            break;
           }
         }
       }
@@ -471,92 +606,149 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       umma_commit(smem_u32(&m->drain));
       wait_bar(smem_u32(&m->drain), 0, m, p.status, false);
     }
-  } else if (warp >= 4 && warp < 8) {
-    // ================= pass-1 consumers: one thread per (query head, window query) row ======
-    const int quad = warp & 3, row = quad * 32 + lane, tid = row;
-    const int t_in_win = row % W;
-    long long n = 0;
-    for (long long idx = blockIdx.x; idx < items1; idx += gridDim.x) {
-      const Item it = decode(p, idx, p.tiles1_per_head, 1);
-      if (!it.valid) continue;
-      const int buf = (int)(n & 1);
-      const bool ok = __all_sync(
-          0xffffffffu, wait_bar(smem_u32(&m->s1_full[buf]), (uint32_t)((n >> 1) & 1), m, p.status));
-      tc_fence_after();
-      // keys this query may see inside the tile: i < n and i <= P + t
-      int limit = 0;
-      if (row < rows_valid) {
-        const int last = min(it.s.n, it.s.prefix + t_in_win + 1);
-        limit = max(0, min(kTile, last - it.tile * kTile));
-      }
-      float mx = -INFINITY, z = 0.f;
-      if (ok) {  // warp-uniform: the TMEM loads below are executed by whole warps
-        const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * 128u;
-        float v[32];
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTile; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-          if (c0 + 32 <= limit) {
+  } else if (warp == 3) {
+    // ================= publisher: chunk statistics leave the CTA; head folding ===============
+    long long j = 0;
+    for (long long c = blockIdx.x; c < total1; c += gridDim.x, ++j) {
+      const Chunk ck = decode_chunk(p, m, c, 1);
+      const int slot = (int)(j & 1);
+      bool ok = true;
+      if (lane == 0)
+        ok = wait_bar(smem_u32(&m->pub_full[slot]), (uint32_t)((j >> 1) & 1), m, p.status);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      float2* dst = p.part + ((size_t)ck.head * p.cph1_max + ck.index) * 128;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) mx = fmaxf(mx, v[c]);
-          } else {
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-              if (c0 + c < limit) mx = fmaxf(mx, v[c]);
-          }
-        }
-        const float m2 = mx * g.scale_log2;
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTile; c0 += 32) {
-          tmem_ld32(taddr + c0, v);
-          if (c0 + 32 <= limit) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) z += fast_exp2(fmaf(v[c], g.scale_log2, -m2));
-          } else {
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-              if (c0 + c < limit) z += fast_exp2(fmaf(v[c], g.scale_log2, -m2));
-          }
-        }
-        mx = m2;
-      }
-      tc_fence_before();
-      mbar_arrive(smem_u32(&m->s1_empty[buf]));
-      ++n;
-      p.part[((size_t)it.head * p.tiles1_per_head + it.tile) * 128 + row] = make_float2(mx, z);
+      for (int q = 0; q < 4; ++q) dst[lane + 32 * q] = m->pub[slot][lane + 32 * q];
       __threadfence();
-      // the value-norm warps have pushed this tile's row norms before the head counter moves
-      if (named_barrier_or(3, 256, m->abort_flag != 0)) break;
-      const int expected = ceil_div(it.s.n, kTile);
-      if (tid == 0) {
-        const int old = atomicAdd(&p.counters[it.head], 1);
-        m->last_flag = (old == expected - 1);
+      __syncwarp();
+      int last = 0;
+      if (lane == 0) {
+        mbar_arrive(smem_u32(&m->pub_empty[slot]));
+        last = atomicAdd(&p.counters[ck.head], 1) == ck.cph - 1;
       }
-      named_barrier(1, 128);
-      const bool last = m->last_flag != 0;
-      named_barrier(1, 128);
+      last = __shfl_sync(0xffffffffu, last, 0);
       if (last) {
         __threadfence();
-        // fold the per-tile partials of this head into one log-sum-exp per window query
-        const float2* pp = p.part + (size_t)it.head * p.tiles1_per_head * 128 + row;
-        float big = -INFINITY, sum = 0.f;
-#pragma unroll 4
-        for (int j = 0; j < expected; ++j) {
-          const float2 pr = __ldcg(pp + (size_t)j * 128);
-          if (pr.y > 0.f) {
-            if (pr.x > big) {
-              sum = sum * fast_exp2(big - pr.x) + pr.y;
-              big = pr.x;
-            } else {
-              sum += pr.y * fast_exp2(pr.x - big);
-            }
-          }
+        // fold the head's chunk partials, in chunk order, into one log-sum-exp per window query
+        const float2* pp = p.part + (size_t)ck.head * p.cph1_max * 128 + lane;
+        float big[4], sum[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          big[q] = -INFINITY;
+          sum[q] = 0.f;
         }
-        p.neg_lse[(size_t)it.head * 128 + row] = sum > 0.f ? -(big + log2f(sum)) : -INFINITY;
+        for (int i0 = 0; i0 < ck.cph; i0 += 8) {
+          float2 pr[8][4];
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              pr[u][q] = (i0 + u < ck.cph) ? __ldcg(pp + (size_t)(i0 + u) * 128 + 32 * q)
+                                           : make_float2(-INFINITY, 0.f);
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float2 v = pr[u][q];
+              if (v.y > 0.f) {
+                if (v.x > big[q]) {
+                  sum[q] = sum[q] * fast_exp2(big[q] - v.x) + v.y;
+                  big[q] = v.x;
+                } else {
+                  sum[q] += v.y * fast_exp2(v.x - big[q]);
+                }
+              }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          p.neg_lse[(size_t)ck.head * 128 + lane + 32 * q] =
+              sum[q] > 0.f ? -(big[q] + log2f(sum[q])) : -INFINITY;
         __threadfence();
-        named_barrier(1, 128);
-        if (tid == 0) st_release(&p.ready[it.head], 1);
+        __syncwarp();
+        if (lane == 0) st_release(&p.ready[ck.head], 1);
       }
+    }
+  } else if (warp >= 4 && warp < 8) {
+    // ================= pass-1 consumers: one thread per (query head, window query) row ======
+    const int quad = warp & 3, row = quad * 32 + lane;
+    const int t_in_win = row % W;
+    const float sc2 = g.scale_log2;
+    long long n = 0, j = 0;
+    bool alive = true;
+    for (long long c = blockIdx.x; c < total1 && alive; c += gridDim.x, ++j) {
+      const Chunk ck = decode_chunk(p, m, c, 1);
+      // keys this query may see: i < n and i <= P + t
+      const int last = row < rows_valid ? min(ck.s.n, ck.s.prefix + t_in_win + 1) : 0;
+      float mx = -INFINITY, z = 0.f;
+      for (int t = 0; t < ck.ntiles; ++t, ++n) {
+        const int buf = (int)(n & 1);
+        alive = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->s1_full[buf]),
+                                                 (uint32_t)((n >> 1) & 1), m, p.status));
+        if (!alive) break;
+        tc_fence_after();
+        const int limit = max(0, min(kTile, last - (ck.tile0 + t) * kTile));
+        const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * 128u;
+        float va[32], vb[32];
+        tmem_ld32_issue(taddr, va);
+        tmem_ld_wait(va);
+#pragma unroll
+        for (int blk = 0; blk < 4; ++blk) {
+          float* cur = (blk & 1) ? vb : va;
+          float* nxt = (blk & 1) ? va : vb;
+          if (blk < 3) tmem_ld32_issue(taddr + (blk + 1) * 32, nxt);
+          const int cnt = limit - blk * 32;
+          if (cnt >= 32) {
+            float b0 = fmaxf(cur[0], cur[1]), b1 = fmaxf(cur[2], cur[3]);
+#pragma unroll
+            for (int i = 4; i < 32; i += 4) {
+              b0 = fmaxf(b0, fmaxf(cur[i], cur[i + 1]));
+              b1 = fmaxf(b1, fmaxf(cur[i + 2], cur[i + 3]));
+            }
+            const float nm = fmaxf(b0, b1) * sc2;
+            if (nm > mx) {
+              z *= fast_exp2(mx - nm);
+              mx = nm;
+            }
+            float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              z0 += fast_exp2(fmaf(cur[i + 0], sc2, -mx));
+              z1 += fast_exp2(fmaf(cur[i + 1], sc2, -mx));
+              z2 += fast_exp2(fmaf(cur[i + 2], sc2, -mx));
+              z3 += fast_exp2(fmaf(cur[i + 3], sc2, -mx));
+            }
+            z += (z0 + z1) + (z2 + z3);
+          } else if (cnt > 0) {
+            float bm = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i < cnt) bm = fmaxf(bm, cur[i]);
+            const float nm = bm * sc2;
+            if (nm > mx) {
+              z *= fast_exp2(mx - nm);
+              mx = nm;
+            }
+            float zz = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i < cnt) zz += fast_exp2(fmaf(cur[i], sc2, -mx));
+            z += zz;
+          }
+          if (blk < 3) tmem_ld_wait(nxt);
+        }
+        tc_fence_before();
+        mbar_arrive(smem_u32(&m->s1_empty[buf]));
+      }
+      if (!alive) break;
+      // hand the chunk's statistics to the publisher warp
+      const int slot = (int)(j & 1);
+      alive = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->pub_empty[slot]),
+                                               (uint32_t)((j >> 1) & 1) ^ 1, m, p.status));
+      if (!alive) break;
+      m->pub[slot][row] = make_float2(mx, z);
+      mbar_arrive(smem_u32(&m->pub_full[slot]));
     }
   } else if (warp >= 8 && warp < 12) {
     // ================= pass-2 consumers: one thread per key ==================================
@@ -564,99 +756,98 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     const int quad = warp & 3, key_lane = quad * 32 + lane, tid = key_lane;
     const int rad = g.pool_radius;
     const float inv_w = 1.0f / (float)W;
-    int cur_head = -1;
-    float head_scale = 0.f;
-    long long n = 0;
-    for (long long idx = blockIdx.x; idx < items2; idx += gridDim.x) {
-      const Item it = decode(p, idx, p.tiles2_per_head, 2);
-      if (!it.valid) continue;
-      if (it.head != cur_head) {
-        if (tid == 0) {
-          m->p2_head = it.head;
-          uint32_t spins = 0;
-          while (ld_acquire(&p.ready[it.head]) == 0) {
-            if (m->abort_flag) break;
-            __nanosleep(64);
-            if (++spins > kSpinLimit) {
-              m->abort_flag = 1;
-              atomicOr(p.status, LAVA_DEV_WAIT_EXPIRED);
-              break;
+    const float sc2 = g.scale_log2;
+    long long n = 0, j = 0;
+    bool alive = true;
+    if (tid == 0 && (long long)blockIdx.x < total2) {
+      const Chunk first = decode_chunk(p, m, blockIdx.x, 2);
+      m->p2_pos = key_pos(p, first.head, (long long)first.tile0 * p.out_keys);
+    }
+    // Exits are taken only after a barrier that ORs the stop condition over all four warps, so
+    // no warp is ever left waiting at a barrier the others have abandoned.
+    for (long long c = blockIdx.x; c < total2 && alive; c += gridDim.x, ++j) {
+      const Chunk ck = decode_chunk(p, m, c, 2);
+      const int slot = (int)(j & 1);
+      const bool got = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->prep_full[slot]),
+                                                        (uint32_t)((j >> 1) & 1), m, p.status));
+      if (named_barrier_or(2, 128, !got || m->abort_flag != 0)) break;
+      const Prep* prep = &m->prep[slot];
+      const float head_scale = prep->scale;
+      float es = 0.f, et = 0.f;  // entropy sums of this thread's keys over the chunk
+      for (int t = 0; t < ck.ntiles; ++t, ++n) {
+        const int tile = ck.tile0 + t;
+        const int buf = (int)(n & 1);
+        const bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->s2_full[buf]),
+                                                         (uint32_t)((n >> 1) & 1), m, p.status));
+        tc_fence_after();
+        float acc[NH];
+#pragma unroll
+        for (int h = 0; h < NH; ++h) acc[h] = 0.f;
+        if (ok) {  // warp-uniform: the TMEM loads below are executed by whole warps
+          const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)buf * 128u;
+          float va[32], vb[32];
+          tmem_ld32_issue(taddr, va);
+          tmem_ld_wait(va);
+#pragma unroll
+          for (int blk = 0; blk < 4; ++blk) {
+            if (blk * 32 < rows_valid) {
+              float* cur = (blk & 1) ? vb : va;
+              float* nxt = (blk & 1) ? va : vb;
+              const bool more = blk < 3 && (blk + 1) * 32 < rows_valid;
+              if (more) tmem_ld32_issue(taddr + (blk + 1) * 32, nxt);
+              const int c0 = blk * 32;
+#pragma unroll
+              for (int c4 = 0; c4 < 32; c4 += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(&prep->lse[c0 + c4]);
+                acc[(c0 + c4 + 0) / W] += fast_exp2(fmaf(cur[c4 + 0], sc2, l4.x));
+                acc[(c0 + c4 + 1) / W] += fast_exp2(fmaf(cur[c4 + 1], sc2, l4.y));
+                acc[(c0 + c4 + 2) / W] += fast_exp2(fmaf(cur[c4 + 2], sc2, l4.z));
+                acc[(c0 + c4 + 3) / W] += fast_exp2(fmaf(cur[c4 + 3], sc2, l4.w));
+              }
+              if (more) tmem_ld_wait(nxt);
             }
           }
+          tc_fence_before();
+          mbar_arrive(smem_u32(&m->s2_empty[buf]));
         }
-        if (named_barrier_or(2, 128, m->abort_flag != 0)) break;
-        m->lse[tid] = __ldcg(p.neg_lse + (size_t)it.head * 128 + tid);
-        const float vb = p.vbar_in ? p.vbar_in[it.head]
-                                   : __uint_as_float(__ldcg(p.vbar_bits + it.head));
-        head_scale = vb * g.c_hat;
-        if (tid == 0 && p.vbar_out) p.vbar_out[it.head] = vb;
-        cur_head = it.head;
-        named_barrier(2, 128);
-      }
-      const int buf = (int)(n & 1);
-      const bool ok = __all_sync(
-          0xffffffffu, wait_bar(smem_u32(&m->s2_full[buf]), (uint32_t)((n >> 1) & 1), m, p.status));
-      tc_fence_after();
-      float acc[NH];
+        const int ab = (int)(n & 1);
 #pragma unroll
-      for (int h = 0; h < NH; ++h) acc[h] = 0.f;
-      if (ok) {
-        const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)buf * 128u;
-        float v[32];
-#pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          if (c0 < rows_valid) {
-            tmem_ld32(taddr + c0, v);
-#pragma unroll
-            for (int c4 = 0; c4 < 32; c4 += 4) {
-              const float4 l4 = *reinterpret_cast<const float4*>(&m->lse[c0 + c4]);
-              acc[(c0 + c4 + 0) / W] += fast_exp2(fmaf(v[c4 + 0], g.scale_log2, l4.x));
-              acc[(c0 + c4 + 1) / W] += fast_exp2(fmaf(v[c4 + 1], g.scale_log2, l4.y));
-              acc[(c0 + c4 + 2) / W] += fast_exp2(fmaf(v[c4 + 2], g.scale_log2, l4.z));
-              acc[(c0 + c4 + 3) / W] += fast_exp2(fmaf(v[c4 + 3], g.scale_log2, l4.w));
+        for (int h = 0; h < NH; ++h) m->a[ab][h][key_lane] = acc[h] * inv_w;
+        if (named_barrier_or(2, 128, !ok || m->abort_flag != 0)) {
+          alive = false;
+          break;
+        }
+        // lane <-> key: the tile starts pool_radius keys before the first key it owns
+        const int key0 = tile * p.out_keys - rad;
+        const int i = key0 + key_lane;
+        const int own_lo = tile * p.out_keys, own_hi = min(ck.s.prefix, own_lo + p.out_keys);
+        if (i >= own_lo && i < own_hi) {
+          const int lo = max(0, i - rad) - key0, hi = min(ck.s.prefix - 1, i + rad) - key0;
+          float best = 0.f;
+          for (int h = 0; h < g.group; ++h) {
+            const float* a = m->a[ab][h];
+            float pv;
+            if (g.pool_kind == LAVA_POOL_AVG) {
+              pv = 0.f;
+              for (int q = lo; q <= hi; ++q) pv += a[q];
+              pv = pv / (float)g.pool_kernel;
+            } else {
+              pv = a[lo];
+              for (int q = lo + 1; q <= hi; ++q) pv = fmaxf(pv, a[q]);
             }
+            best = fmaxf(best, pv);
+          }
+          const float sc = best * head_scale;
+          p.scores[(size_t)ck.layer * g.total_scores + ck.s.score_off +
+                   (long long)ck.kvh * ck.s.prefix + i] = sc;
+          if (sc > 0.f) {
+            es += sc;
+            et += sc * logf(sc);
           }
         }
       }
-      tc_fence_before();
-      mbar_arrive(smem_u32(&m->s2_empty[buf]));
-      const int ab = (int)(n & 1);
-      ++n;
-#pragma unroll
-      for (int h = 0; h < NH; ++h) m->a[ab][h][key_lane] = acc[h] * inv_w;
-      if (named_barrier_or(2, 128, m->abort_flag != 0)) break;
-      // lane <-> key: the tile starts pool_radius keys before the first key it owns
-      const int key0 = it.tile * p.out_keys - rad;
-      const int i = key0 + key_lane;
-      const int own_lo = it.tile * p.out_keys, own_hi = min(it.s.prefix, own_lo + p.out_keys);
-      float sc = 0.f;
-      const bool mine = i >= own_lo && i < own_hi;
-      if (mine) {
-        const int lo = max(0, i - rad) - key0, hi = min(it.s.prefix - 1, i + rad) - key0;
-        float best = 0.f;
-        for (int h = 0; h < g.group; ++h) {
-          const float* a = m->a[ab][h];
-          float pv;
-          if (g.pool_kind == LAVA_POOL_AVG) {
-            pv = 0.f;
-            for (int j = lo; j <= hi; ++j) pv += a[j];
-            pv = pv / (float)g.pool_kernel;
-          } else {
-            pv = a[lo];
-            for (int j = lo + 1; j <= hi; ++j) pv = fmaxf(pv, a[j]);
-          }
-          best = fmaxf(best, pv);
-        }
-        sc = best * head_scale;
-        p.scores[(size_t)it.layer * g.total_scores + it.s.score_off +
-                 (long long)it.kvh * it.s.prefix + i] = sc;
-      }
-      // entropy sums of this tile in a fixed order: lanes, then warps
-      float es = 0.f, et = 0.f;
-      if (mine && sc > 0.f) {
-        es = sc;
-        et = sc * logf(sc);
-      }
+      if (!alive) break;
+      // entropy sums of the chunk in a fixed order: keys of a thread, lanes, then warps
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         es += __shfl_down_sync(0xffffffffu, es, o);
@@ -672,53 +863,61 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
                              ((double)m->red[0][2] + (double)m->red[0][3]);
         const double t_sum = ((double)m->red[1][0] + (double)m->red[1][1]) +
                              ((double)m->red[1][2] + (double)m->red[1][3]);
-        p.ent_part[(size_t)it.head * p.tiles2_per_head + it.tile] = make_double2(s_sum, t_sum);
-      }
-    }
-    if (tid == 0) m->p2_head = 0x3fffffff;  // pass 1 is no longer held back
-  } else if (warp >= 12) {
-    // ================= value-norm warps: rows of V that belong to the pass-1 tile ============
-    const int vt = threadIdx.x - 12 * 32;       // 0..127
-    const int sub = vt >> 4, piece = vt & 15;   // 8 rows at a time, 16 x 16 B per row
-    for (long long idx = blockIdx.x; idx < items1; idx += gridDim.x) {
-      const Item it = decode(p, idx, p.tiles1_per_head, 1);
-      if (!it.valid) continue;
-      if (!p.vbar_in) {
-        const int row0 = it.tile * kTile;
-        const char* vb = p.v + ((size_t)it.layer * p.v_ls + (long long)it.kvh * g.v_sh) * 2;
-        uint4 raw[16];
-#pragma unroll
-        for (int r = 0; r < 16; ++r) {
-          const int row = row0 + r * 8 + sub;
-          raw[r] = make_uint4(0, 0, 0, 0);
-          if (row < it.s.n) {
-            const uint4* src = reinterpret_cast<const uint4*>(
-                vb + (it.s.tok0 + row) * g.v_st * 2 + piece * 16);
-            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(raw[r].x), "=r"(raw[r].y), "=r"(raw[r].z), "=r"(raw[r].w)
-                         : "l"(src));
-          }
+        p.ent_part[(size_t)ck.head * p.cph2_max + ck.index] = make_double2(s_sum, t_sum);
+        mbar_arrive(smem_u32(&m->prep_empty[slot]));
+        // the throttle of pass 1 follows the first key this CTA has still to score
+        long long next = 0x3fffffffffffffffLL;
+        if (c + gridDim.x < total2) {
+          const Chunk nx = decode_chunk(p, m, c + gridDim.x, 2);
+          next = key_pos(p, nx.head, (long long)nx.tile0 * p.out_keys);
         }
+        m->p2_pos = next;
+      }
+      named_barrier(2, 128);  // red[] is free again
+    }
+    if (tid == 0) m->p2_pos = 0x3fffffffffffffffLL;  // pass 1 is no longer held back
+  } else {
+    // ================= value-norm warps: the V rows of the CTA's pass-1 chunks ===============
+    if (!p.vbar_in) {
+      const uint64_t drop = policy_evict_first();
+      const int vt = threadIdx.x - 12 * 32;       // 0..127
+      const int sub = vt >> 4, piece = vt & 15;   // 8 rows at a time, 16 x 16 B per row
+      for (long long c = blockIdx.x; c < total1 && !m->abort_flag; c += gridDim.x) {
+        const Chunk ck = decode_chunk(p, m, c, 1);
+        const int row_lo = ck.tile0 * kTile, row_hi = min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile);
+        const char* vb = p.v + ((size_t)ck.layer * p.v_ls + (long long)ck.kvh * g.v_sh) * 2 +
+                         piece * 16;
         float best = 0.f;
+        for (int r0 = row_lo; r0 < row_hi; r0 += 128) {
+          uint4 raw[16];
 #pragma unroll
-        for (int r = 0; r < 16; ++r) {
-          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw[r]);
-          float sum = 0.f;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float2 f = __bfloat1622float2(h2[j]);
-            sum += fabsf(f.x) + fabsf(f.y);
+          for (int r = 0; r < 16; ++r) {
+            const int row = r0 + r * 8 + sub;
+            raw[r] = make_uint4(0, 0, 0, 0);
+            if (row < row_hi) raw[r] = ld_stream16(vb + (ck.s.tok0 + row) * g.v_st * 2, drop);
           }
 #pragma unroll
-          for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-          best = fmaxf(best, sum);
+          for (int r = 0; r < 16; ++r) {
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw[r]);
+            float sum = 0.f;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float2 f = __bfloat1622float2(h2[q]);
+              sum += fabsf(f.x) + fabsf(f.y);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            best = fmaxf(best, sum);
+          }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
-        if (lane == 0) atomicMax(&p.vbar_bits[it.head], __float_as_uint(best));
-        __threadfence();
+        if (lane == 0) {
+          atomicMax(&p.vbar_bits[ck.head], __float_as_uint(best));
+          __threadfence();
+          atomicAdd(&p.vcount[ck.head], 1);
+        }
       }
-      if (named_barrier_or(3, 256, m->abort_flag != 0)) break;
     }
   }
 
@@ -729,19 +928,24 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
   if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
-// entropy of one (layer, sequence) from the per-tile sums, folded in a fixed order
+// entropy of one (layer, sequence) from the per-chunk sums, folded in a fixed order
 __global__ void __launch_bounds__(256)
-entropy_finalize_sm100_kernel(Geom g, const double2* ent_part, int tiles2_per_head, int out_keys,
-                              double* entropy) {
+entropy_finalize_sm100_kernel(Geom g, const double2* ent_part, int cph2_max, int chunk_keys,
+                              double* entropy, const float* vbar_in, const unsigned* vbar_bits,
+                              float* vbar_out) {
   __shared__ double rs[8], rt[8];
   const int prob = blockIdx.x, layer = prob / g.batch, b = prob - layer * g.batch;
   const SeqInfo s = seq_info(g, b);
-  const int used = ceil_div(s.prefix, out_keys);
+  const int used = ceil_div(s.prefix, chunk_keys);
   const int total = g.n_kv_heads * used;
+  if (vbar_out && (int)threadIdx.x < g.n_kv_heads) {
+    const size_t head = (size_t)prob * g.n_kv_heads + threadIdx.x;
+    vbar_out[head] = vbar_in ? vbar_in[head] : __uint_as_float(vbar_bits[head]);
+  }
   double sum_s = 0.0, sum_t = 0.0;
   for (int i = threadIdx.x; i < total; i += 256) {
     const int kvh = i / used, t = i - kvh * used;
-    const double2 v = ent_part[((size_t)prob * g.n_kv_heads + kvh) * tiles2_per_head + t];
+    const double2 v = ent_part[((size_t)prob * g.n_kv_heads + kvh) * cph2_max + t];
     sum_s += v.x;
     sum_t += v.y;
   }
@@ -790,6 +994,17 @@ EncodeTiledFn encode_fn() {
 
 size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
+// tiles per chunk: tuning knob (LAVA_SM100_CHUNK_TILES), default 4
+int chunk_tiles_setting() {
+  static int value = 0;
+  if (!value) {
+    const char* e = getenv("LAVA_SM100_CHUNK_TILES");
+    const int v = e ? atoi(e) : 0;
+    value = (v >= 1 && v <= 64) ? v : 4;
+  }
+  return value;
+}
+
 }  // namespace
 
 bool sm100_supported(const Geom& g) {
@@ -797,18 +1012,20 @@ bool sm100_supported(const Geom& g) {
   if (g.window != 16 && g.window != 32 && g.window != 64 && g.window != 128) return false;
   if (g.group * g.window > 128 || g.group > 8) return false;
   if (g.pool_radius > 31) return false;
+  if (g.batch > kMaxBatch) return false;
   return true;
 }
 
 Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   Sm100Layout l;
+  const int r = chunk_tiles_setting();
   l.heads_total = n_layers * g.batch * g.n_kv_heads;
-  l.tiles1 = ceil_div(g.max_seqlen, kTile);
   l.out_keys = kTile - 2 * g.pool_radius;
-  l.tiles2 = ceil_div(max(1, g.max_seqlen - g.window), l.out_keys);
+  l.tiles1 = ceil_div(ceil_div(g.max_seqlen, kTile), r);                       // chunks, pass 1
+  l.tiles2 = ceil_div(ceil_div(max(1, g.max_seqlen - g.window), l.out_keys), r);  // chunks, pass 2
   size_t off = 0;
-  l.off_sync = off;   // counters, ready flags, value-norm bits: zeroed before every launch
-  off = up256(off + sizeof(int) * 3 * (size_t)l.heads_total);
+  l.off_sync = off;   // counters, ready flags, value-norm counters and bits: zeroed every launch
+  off = up256(off + sizeof(int) * 4 * (size_t)l.heads_total);
   l.sync_bytes = off;
   l.off_part = off;
   off = up256(off + sizeof(float2) * 128 * (size_t)l.heads_total * l.tiles1);
@@ -856,17 +1073,22 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
       return fail(LAVA_ERR_CUDA, "tensor map for K could not be encoded");
   }
 
+  int dev = 0, sms = 0;
+  lava_status rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+  if (rc != LAVA_OK) return rc;
+  rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "SM count");
+  if (rc != LAVA_OK) return rc;
+
   Sm100Params p;
   p.g = g;
   p.n_layers = n_layers;
-  p.heads_total = lay.heads_total;
-  p.tiles1_per_head = lay.tiles1;
-  p.tiles2_per_head = lay.tiles2;
+  p.chunk_tiles = chunk_tiles_setting();
   p.out_keys = lay.out_keys;
-  // keep pass 1 within roughly 32 MiB of K+V traffic of pass 2
-  const double head_bytes = 2.0 * (double)g.max_seqlen * 256.0;
-  int lag = (int)(32.0 * 1024 * 1024 / head_bytes);
-  p.lag_heads = lag < 1 ? 1 : (lag > 64 ? 64 : lag);
+  p.cph1_max = lay.tiles1;
+  p.cph2_max = lay.tiles2;
+  // Pass 1 must be allowed to finish the head pass 2 is waiting for (one head = max_seqlen
+  // keys); two further rounds of chunks cover the time the head's statistics take to fold.
+  p.lag_keys = (long long)g.max_seqlen + 2LL * sms * p.chunk_tiles * kTile;
   p.vbar_in = vbar_in;
   p.scores = scores;
   p.vbar_out = vbar_out;
@@ -874,20 +1096,15 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.v_ls = v_ls;
   p.counters = reinterpret_cast<int*>(ws + lay.off_sync);
   p.ready = p.counters + lay.heads_total;
-  p.vbar_bits = reinterpret_cast<unsigned*>(p.ready + lay.heads_total);
+  p.vcount = p.ready + lay.heads_total;
+  p.vbar_bits = reinterpret_cast<unsigned*>(p.vcount + lay.heads_total);
   p.part = reinterpret_cast<float2*>(ws + lay.off_part);
   p.neg_lse = reinterpret_cast<float*>(ws + lay.off_lse);
   p.ent_part = reinterpret_cast<double2*>(ws + lay.off_ent);
   p.status = reinterpret_cast<unsigned*>(ws_base);  // the status word opens the workspace
 
-  lava_status rc = check_cuda(cudaMemsetAsync(ws + lay.off_sync, 0, lay.sync_bytes, stream),
-                              "sync scratch clear");
-  if (rc != LAVA_OK) return rc;
-
-  int dev = 0, sms = 0;
-  rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
-  if (rc != LAVA_OK) return rc;
-  rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "SM count");
+  rc = check_cuda(cudaMemsetAsync(ws + lay.off_sync, 0, lay.sync_bytes, stream),
+                  "sync scratch clear");
   if (rc != LAVA_OK) return rc;
 
   void (*kern)(const CUtensorMap, const CUtensorMap, const Sm100Params) = nullptr;
@@ -900,13 +1117,17 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   rc = check_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)kSmemBytes), "cudaFuncSetAttribute(sm100 score)");
   if (rc != LAVA_OK) return rc;
-  const long long items = (long long)lay.heads_total * lay.tiles1;
-  const int grid = (int)(items < sms ? items : sms);
-  kern<<<grid, kThreads, kSmemBytes, stream>>>(map_q, map_k, p);
-  rc = check_cuda(cudaGetLastError(), "score (sm100) launch");
+  // an upper bound on the pass-1 chunks; CTAs beyond the real count find no work and exit
+  const long long chunks = (long long)lay.heads_total * lay.tiles1;
+  const int grid = (int)(chunks < sms ? chunks : sms);
+  // Cooperative launch: the CTAs wait on one another's flags, so all must be resident at once.
+  void* args[3] = {&map_q, &map_k, &p};
+  rc = check_cuda(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args,
+                                              kSmemBytes, stream), "score (sm100) launch");
   if (rc != LAVA_OK) return rc;
   entropy_finalize_sm100_kernel<<<n_layers * g.batch, 256, 0, stream>>>(
-      g, p.ent_part, lay.tiles2, lay.out_keys, entropy);
+      g, p.ent_part, lay.tiles2, p.chunk_tiles * lay.out_keys, entropy, vbar_in, p.vbar_bits,
+      vbar_out);
   count_launches(2);
   return check_cuda(cudaGetLastError(), "entropy finalize launch");
 }
