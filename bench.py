@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run only the first N layers of the workload (small cases for profiling; "
+                         "the budget shrinks in proportion and the line says so)")
     return ap.parse_args()
 
 
@@ -230,6 +233,8 @@ def main():
     lava.load_library()
 
     cfg = get_config(args.workload)
+    if args.layers > 0:
+        cfg = cfg.scaled(n_layers=min(args.layers, cfg.n_layers))
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     L, hkv, hq, d, w, T = (cfg.n_layers, cfg.n_kv_heads, cfg.n_q_heads, cfg.head_dim, cfg.window,

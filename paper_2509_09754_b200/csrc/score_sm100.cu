@@ -30,7 +30,8 @@ namespace lava {
 namespace {
 
 constexpr int kTile = 128;           // keys per tile
-constexpr int kThreads = 512;        // 16 warps
+constexpr int kThreads = 640;        // 20 warps: 4 service, 4 + 4 consumer, 8 value-norm
+constexpr int kVWarps = 8;
 constexpr int kStages = 2;           // K stages per pipeline
 constexpr int kMaxBatch = 512;       // sequences the in-kernel chunk schedule can index
 constexpr uint32_t kTileBytes = 128 * 128 * 2;  // one [128 x 128] bf16 tile = 2 swizzled blocks
@@ -468,7 +469,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       // wait until the head's log-sum-exp and value norm are final
       bool ok = true;
       if (lane == 0) {
-        const int want_v = p.vbar_in ? 0 : 4 * ceil_div(ceil_div(ck.s.n, kTile), p.chunk_tiles);
+        const int want_v = p.vbar_in ? 0 : kVWarps * ceil_div(ceil_div(ck.s.n, kTile), p.chunk_tiles);
         uint32_t spins = 0;
         while (ld_acquire(&p.ready[ck.head]) == 0 ||
                (want_v && ld_acquire(&p.vcount[ck.head]) < want_v)) {
@@ -690,15 +691,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         tc_fence_after();
         const int limit = max(0, min(kTile, last - (ck.tile0 + t) * kTile));
         const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * 128u;
-        float va[32], vb[32];
-        tmem_ld32_issue(taddr, va);
-        tmem_ld_wait(va);
-#pragma unroll
+        // a compact loop body: the four warp roles of a scheduler share its instruction cache
+#pragma unroll 1
         for (int blk = 0; blk < 4; ++blk) {
-          float* cur = (blk & 1) ? vb : va;
-          float* nxt = (blk & 1) ? va : vb;
-          if (blk < 3) tmem_ld32_issue(taddr + (blk + 1) * 32, nxt);
           const int cnt = limit - blk * 32;
+          float cur[32];
+          tmem_ld32_issue(taddr + blk * 32, cur);
+          tmem_ld_wait(cur);
           if (cnt >= 32) {
             float b0 = fmaxf(cur[0], cur[1]), b1 = fmaxf(cur[2], cur[3]);
 #pragma unroll
@@ -736,7 +735,6 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
               if (i < cnt) zz += fast_exp2(fmaf(cur[i], sc2, -mx));
             z += zz;
           }
-          if (blk < 3) tmem_ld_wait(nxt);
         }
         tc_fence_before();
         mbar_arrive(smem_u32(&m->s1_empty[buf]));
@@ -785,64 +783,100 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         for (int h = 0; h < NH; ++h) acc[h] = 0.f;
         if (ok) {  // warp-uniform: the TMEM loads below are executed by whole warps
           const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)buf * 128u;
-          float va[32], vb[32];
-          tmem_ld32_issue(taddr, va);
-          tmem_ld_wait(va);
-#pragma unroll
-          for (int blk = 0; blk < 4; ++blk) {
-            if (blk * 32 < rows_valid) {
-              float* cur = (blk & 1) ? vb : va;
-              float* nxt = (blk & 1) ? va : vb;
-              const bool more = blk < 3 && (blk + 1) * 32 < rows_valid;
-              if (more) tmem_ld32_issue(taddr + (blk + 1) * 32, nxt);
-              const int c0 = blk * 32;
+          // window queries come in blocks of 32 columns; a block never straddles two query
+          // heads when W >= 32, and covers 32 / W whole heads otherwise
+          const int nblk = (rows_valid + 31) >> 5;
+#pragma unroll 1
+          for (int blk = 0; blk < nblk; ++blk) {
+            float cur[32];
+            tmem_ld32_issue(taddr + blk * 32, cur);
+            tmem_ld_wait(cur);
+            const float* lse = &prep->lse[blk * 32];
+            if (W >= 32) {
+              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
               for (int c4 = 0; c4 < 32; c4 += 4) {
-                const float4 l4 = *reinterpret_cast<const float4*>(&prep->lse[c0 + c4]);
-                acc[(c0 + c4 + 0) / W] += fast_exp2(fmaf(cur[c4 + 0], sc2, l4.x));
-                acc[(c0 + c4 + 1) / W] += fast_exp2(fmaf(cur[c4 + 1], sc2, l4.y));
-                acc[(c0 + c4 + 2) / W] += fast_exp2(fmaf(cur[c4 + 2], sc2, l4.z));
-                acc[(c0 + c4 + 3) / W] += fast_exp2(fmaf(cur[c4 + 3], sc2, l4.w));
+                const float4 l4 = *reinterpret_cast<const float4*>(lse + c4);
+                s0 += fast_exp2(fmaf(cur[c4 + 0], sc2, l4.x));
+                s1 += fast_exp2(fmaf(cur[c4 + 1], sc2, l4.y));
+                s2 += fast_exp2(fmaf(cur[c4 + 2], sc2, l4.z));
+                s3 += fast_exp2(fmaf(cur[c4 + 3], sc2, l4.w));
               }
-              if (more) tmem_ld_wait(nxt);
+              const float sum = (s0 + s1) + (s2 + s3);
+              const int h = (blk * 32) / W;
+#pragma unroll
+              for (int hh = 0; hh < NH; ++hh)
+                if (hh == h) acc[hh] += sum;
+            } else {  // W == 16: two query heads per block
+              float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+              for (int c4 = 0; c4 < 16; c4 += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(lse + c4);
+                const float4 r4 = *reinterpret_cast<const float4*>(lse + 16 + c4);
+                s0 += (fast_exp2(fmaf(cur[c4 + 0], sc2, l4.x)) + fast_exp2(fmaf(cur[c4 + 1], sc2, l4.y))) +
+                      (fast_exp2(fmaf(cur[c4 + 2], sc2, l4.z)) + fast_exp2(fmaf(cur[c4 + 3], sc2, l4.w)));
+                s1 += (fast_exp2(fmaf(cur[16 + c4 + 0], sc2, r4.x)) + fast_exp2(fmaf(cur[16 + c4 + 1], sc2, r4.y))) +
+                      (fast_exp2(fmaf(cur[16 + c4 + 2], sc2, r4.z)) + fast_exp2(fmaf(cur[16 + c4 + 3], sc2, r4.w)));
+              }
+#pragma unroll
+              for (int hh = 0; hh < NH; hh += 2)
+                if (hh == 2 * blk) {
+                  acc[hh] += s0;
+                  if (hh + 1 < NH) acc[hh + 1] += s1;
+                }
             }
           }
           tc_fence_before();
           mbar_arrive(smem_u32(&m->s2_empty[buf]));
         }
+        // lane <-> key: the tile starts pool_radius keys before the first key it owns; keys
+        // outside the prefix hold the neutral element of both pools (values are >= 0)
         const int ab = (int)(n & 1);
+        const int key0 = tile * p.out_keys - rad;
+        const int i = key0 + key_lane;
+        const bool inside = i >= 0 && i < ck.s.prefix;
+        const bool avg = g.pool_kind == LAVA_POOL_AVG;
+        if (avg) {
 #pragma unroll
-        for (int h = 0; h < NH; ++h) m->a[ab][h][key_lane] = acc[h] * inv_w;
+          for (int h = 0; h < NH; ++h) m->a[ab][h][key_lane] = inside ? acc[h] * inv_w : 0.f;
+        } else {
+          // max-pooling commutes with the group maximum: reduce over the query heads first
+          float top = 0.f;
+#pragma unroll
+          for (int h = 0; h < NH; ++h)
+            if (h < g.group) top = fmaxf(top, acc[h] * inv_w);
+          m->a[ab][0][key_lane] = inside ? top : 0.f;
+        }
         if (named_barrier_or(2, 128, !ok || m->abort_flag != 0)) {
           alive = false;
           break;
         }
-        // lane <-> key: the tile starts pool_radius keys before the first key it owns
-        const int key0 = tile * p.out_keys - rad;
-        const int i = key0 + key_lane;
         const int own_lo = tile * p.out_keys, own_hi = min(ck.s.prefix, own_lo + p.out_keys);
         if (i >= own_lo && i < own_hi) {
-          const int lo = max(0, i - rad) - key0, hi = min(ck.s.prefix - 1, i + rad) - key0;
           float best = 0.f;
-          for (int h = 0; h < g.group; ++h) {
-            const float* a = m->a[ab][h];
-            float pv;
-            if (g.pool_kind == LAVA_POOL_AVG) {
-              pv = 0.f;
-              for (int q = lo; q <= hi; ++q) pv += a[q];
-              pv = pv / (float)g.pool_kernel;
-            } else {
-              pv = a[lo];
-              for (int q = lo + 1; q <= hi; ++q) pv = fmaxf(pv, a[q]);
+          if (avg) {
+            for (int h = 0; h < g.group; ++h) {
+              const float* a = &m->a[ab][h][key_lane];
+              float pv = 0.f;
+              for (int q = -rad; q <= rad; ++q) pv += a[q];
+              best = fmaxf(best, pv / (float)g.pool_kernel);
             }
-            best = fmaxf(best, pv);
+          } else {
+            const float* a = &m->a[ab][0][key_lane];
+            if (rad == 3) {
+              best = fmaxf(fmaxf(fmaxf(a[-3], a[-2]), fmaxf(a[-1], a[0])),
+                           fmaxf(fmaxf(a[1], a[2]), a[3]));
+            } else {
+              best = a[0];
+              for (int q = 1; q <= rad; ++q) best = fmaxf(best, fmaxf(a[-q], a[q]));
+            }
           }
           const float sc = best * head_scale;
           p.scores[(size_t)ck.layer * g.total_scores + ck.s.score_off +
                    (long long)ck.kvh * ck.s.prefix + i] = sc;
           if (sc > 0.f) {
             es += sc;
-            et += sc * logf(sc);
+            et += sc * __logf(sc);
           }
         }
       }
@@ -878,45 +912,94 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     if (tid == 0) m->p2_pos = 0x3fffffffffffffffLL;  // pass 1 is no longer held back
   } else {
     // ================= value-norm warps: the V rows of the CTA's pass-1 chunks ===============
+    // 256 threads, 16 per row.  Rows are taken in groups of 128 (8 loads of 16 B per thread);
+    // one group is in flight while the previous one is reduced, across chunk borders too.
     if (!p.vbar_in) {
       const uint64_t drop = policy_evict_first();
-      const int vt = threadIdx.x - 12 * 32;       // 0..127
-      const int sub = vt >> 4, piece = vt & 15;   // 8 rows at a time, 16 x 16 B per row
-      for (long long c = blockIdx.x; c < total1 && !m->abort_flag; c += gridDim.x) {
-        const Chunk ck = decode_chunk(p, m, c, 1);
-        const int row_lo = ck.tile0 * kTile, row_hi = min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile);
-        const char* vb = p.v + ((size_t)ck.layer * p.v_ls + (long long)ck.kvh * g.v_sh) * 2 +
-                         piece * 16;
-        float best = 0.f;
-        for (int r0 = row_lo; r0 < row_hi; r0 += 128) {
-          uint4 raw[16];
-#pragma unroll
-          for (int r = 0; r < 16; ++r) {
-            const int row = r0 + r * 8 + sub;
-            raw[r] = make_uint4(0, 0, 0, 0);
-            if (row < row_hi) raw[r] = ld_stream16(vb + (ck.s.tok0 + row) * g.v_st * 2, drop);
-          }
-#pragma unroll
-          for (int r = 0; r < 16; ++r) {
-            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw[r]);
-            float sum = 0.f;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float2 f = __bfloat1622float2(h2[q]);
-              sum += fabsf(f.x) + fabsf(f.y);
-            }
-#pragma unroll
-            for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            best = fmaxf(best, sum);
-          }
+      const int vt = threadIdx.x - 12 * 32;       // 0..255
+      const int sub = vt >> 4, piece = vt & 15;
+      struct Group {
+        const char* base;  // this thread's 16 bytes of row 0 of the sequence
+        int row0, row_hi, head;
+        bool last;         // last group of its chunk
+      };
+      long long c = blockIdx.x;
+      Chunk ck;
+      int grp = 0, ngrp = 0;
+      auto next_group = [&](Group& gr) -> bool {
+        while (grp == ngrp) {
+          if (c >= total1 || m->abort_flag) return false;
+          ck = decode_chunk(p, m, c, 1);
+          c += gridDim.x;
+          grp = 0;
+          ngrp = ceil_div(min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile) - ck.tile0 * kTile, 128);
         }
+        gr.base = p.v + ((size_t)ck.layer * p.v_ls + (long long)ck.kvh * g.v_sh +
+                         ck.s.tok0 * g.v_st) * 2 + piece * 16;
+        gr.row0 = ck.tile0 * kTile + grp * 128 + sub;
+        gr.row_hi = min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile);
+        gr.head = ck.head;
+        gr.last = ++grp == ngrp;
+        return true;
+      };
+      auto issue = [&](uint4 (&buf)[8], const Group& gr) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
-        if (lane == 0) {
-          atomicMax(&p.vbar_bits[ck.head], __float_as_uint(best));
-          __threadfence();
-          atomicAdd(&p.vcount[ck.head], 1);
+        for (int s8 = 0; s8 < 8; ++s8) {
+          const int row = gr.row0 + s8 * 16;
+          buf[s8] = make_uint4(0, 0, 0, 0);
+          if (row < gr.row_hi) buf[s8] = ld_stream16(gr.base + (long long)row * g.v_st * 2, drop);
         }
+      };
+      float best = 0.f;
+      auto reduce = [&](const uint4 (&buf)[8], const Group& gr) {
+        float ps[8];
+#pragma unroll
+        for (int s8 = 0; s8 < 8; ++s8) {
+          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&buf[s8]);
+          float sum = 0.f;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float2 f = __bfloat1622float2(h2[q]);
+            sum += fabsf(f.x) + fabsf(f.y);
+          }
+          ps[s8] = sum;
+        }
+        // eight row sums over the 16 lanes of a row in 8 shuffles: every step halves the rows
+        // a lane still carries and doubles the lanes folded into them
+        const bool b3 = (lane & 8) != 0, b2 = (lane & 4) != 0, b1 = (lane & 2) != 0;
+        float k4[4], k2[2];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          k4[q] = (b3 ? ps[q + 4] : ps[q]) + __shfl_xor_sync(0xffffffffu, b3 ? ps[q] : ps[q + 4], 8);
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+          k2[q] = (b2 ? k4[q + 2] : k4[q]) + __shfl_xor_sync(0xffffffffu, b2 ? k4[q] : k4[q + 2], 4);
+        float k1 = (b1 ? k2[1] : k2[0]) + __shfl_xor_sync(0xffffffffu, b1 ? k2[0] : k2[1], 2);
+        k1 += __shfl_xor_sync(0xffffffffu, k1, 1);
+        best = fmaxf(best, k1);
+        if (gr.last) {  // warp-uniform
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
+          if (lane == 0) {
+            atomicMax(&p.vbar_bits[gr.head], __float_as_uint(best));
+            __threadfence();
+            atomicAdd(&p.vcount[gr.head], 1);
+          }
+          best = 0.f;
+        }
+      };
+      uint4 bufa[8], bufb[8];
+      Group ga, gb;
+      bool have_a = next_group(ga), have_b = false;
+      if (have_a) issue(bufa, ga);
+      while (have_a) {
+        have_b = next_group(gb);
+        if (have_b) issue(bufb, gb);
+        reduce(bufa, ga);
+        if (!have_b) break;
+        have_a = next_group(ga);
+        if (have_a) issue(bufa, ga);
+        reduce(bufb, gb);
       }
     }
   }
