@@ -9,18 +9,22 @@
 //       keys the query may see (Sec. 2: softmax over i <= j).  Work is dealt to CTAs in chunks
 //       of a few consecutive tiles of one head; a chunk's statistics leave the CTA once, through
 //       a publisher warp.  The publisher that completes a head folds the chunk partials, in
-//       chunk order, into one log-sum-exp per query and raises the head's ready flag.  Four more
-//       warps stream the chunk's V rows for the value norm (Theorem 1: max_k ||V[k]||_1).
+//       chunk order, into one log-sum-exp per query and raises the head's ready flag.  Seven
+//       more warps stream the chunk's V rows for the value norm (Theorem 1: max_k ||V[k]||_1).
 //   pass 2 (scores)      S^T = K Q_g^T (rows = keys, columns = window queries)
 //       one thread per key: a_h[i] = (1/w) sum_t exp2(z - lse_t) per query head in registers,
 //       pooled over the token axis through shared memory, scaled by Vbar * c_hat, reduced with
 //       the GQA group maximum, written once; entropy sums go to ordered per-chunk slots
 //       (Definition 1, Sec. 4.2, Sec. 4.3, Sec. 5.1 pooling).
 //
+// The exponential unit bounds the kernel, so the eight consumer warps are not split by pass:
+// two groups of four warps each own one TMEM buffer of BOTH pipelines and take whichever of
+// their tiles is ready, which keeps two exp-issuing warps on every scheduler.
+//
 // K is read from HBM once: pass 2 trails pass 1 by a bounded number of keys, so its tiles are
 // still in L2 (K tiles are loaded with an evict-last hint in pass 1 and evict-first in pass 2,
-// V rows with evict-first).  Every wait (mbarrier, ready flag, throttle) is bounded; on expiry
-// the kernel sets LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
+// V rows with evict-first).  Every wait (mbarrier, ready flag, throttle) is bounded in time; on
+// expiry the kernel sets LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -30,13 +34,16 @@ namespace lava {
 namespace {
 
 constexpr int kTile = 128;           // keys per tile
-constexpr int kThreads = 640;        // 20 warps: 4 service, 4 + 4 consumer, 8 value-norm
-constexpr int kVWarps = 8;
+constexpr int kThreads = 640;        // 20 warps: 5 service, 8 consumer, 7 value-norm
+constexpr int kVWarps = 7;
+constexpr int kVRows = kVWarps * 2;  // V rows per load step (16 threads per row)
+constexpr int kMma2Warp = 19;        // issues the pass-2 MMAs (warp 2 issues pass 1)
 constexpr int kStages = 2;           // K stages per pipeline
 constexpr int kMaxBatch = 512;       // sequences the in-kernel chunk schedule can index
 constexpr uint32_t kTileBytes = 128 * 128 * 2;  // one [128 x 128] bf16 tile = 2 swizzled blocks
 constexpr uint32_t kHalfBytes = kTileBytes / 2;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr long long kWaitCycles = 1ll << 32;  // every wait gives up after about two seconds
+constexpr unsigned kBackoffNs = 40;           // pause of a consumer group that found no tile ready
 
 // shared memory map (bytes from a 1024-aligned base)
 constexpr uint32_t kOffQ1 = 0;
@@ -44,7 +51,7 @@ constexpr uint32_t kOffQ2 = kOffQ1 + kTileBytes;
 constexpr uint32_t kOffK1 = kOffQ2 + kTileBytes;
 constexpr uint32_t kOffK2 = kOffK1 + kStages * kTileBytes;
 constexpr uint32_t kOffMisc = kOffK2 + kStages * kTileBytes;  // 192 KB
-constexpr uint32_t kMiscBytes = 20480;
+constexpr uint32_t kMiscBytes = 26624;
 constexpr uint32_t kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + alignment slack
 
 struct Prep {                 // what the score warps need to know about a head
@@ -58,15 +65,16 @@ struct Misc {
   unsigned long long q1_full, q1_empty, q2_full, q2_empty;
   unsigned long long s1_full[2], s1_empty[2], s2_full[2], s2_empty[2];
   unsigned long long pub_full[2], pub_empty[2], prep_full[2], prep_empty[2];
-  unsigned long long drain;
+  unsigned long long gsync[2];        // rendezvous of the four warps of a consumer group
+  unsigned long long drain, drain2;
   volatile long long p2_pos;  // first key (global key coordinate) pass 2 has not finished yet
   uint32_t tmem_base;
   volatile int abort_flag;
   int sched_total1, sched_total2;     // chunks per layer of pass 1 / pass 2
-  alignas(16) float2 pub[2][128];     // (max, sum) of a finished pass-1 chunk, per window query
+  alignas(16) float pub[2][2][128];   // [slot][group][query]: log2-sum-exp of a finished chunk
   Prep prep[2];
-  alignas(16) float a[2][8][kTile];   // window-mean attention per (query head, key) of a tile
-  float red[2][4];
+  alignas(16) float a[2][2][8][kTile];  // [group][tile parity][query head][key]: window means
+  float red[2][2][4];                 // [group][S or T][warp]
   int pref1[kMaxBatch + 1], pref2[kMaxBatch + 1];  // exclusive scans of chunks per sequence
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
@@ -84,13 +92,13 @@ struct Sm100Params {
   const char* v;
   long long v_ls;
   // scratch
-  float2* part;             // [heads_total][cph1_max][128]
+  float* part;              // [heads_total][cph1_max][128] log2-sum-exp per chunk and query
   int* counters;            // [heads_total] published pass-1 chunks
   int* ready;               // [heads_total]
   int* vcount;              // [heads_total] finished value-norm warps
   unsigned* vbar_bits;      // [heads_total]
   float* neg_lse;           // [heads_total][128]
-  double2* ent_part;        // [heads_total][cph2_max]
+  double2* ent_part;        // [heads_total][cph2_max][2 consumer groups]
   unsigned* status;
 };
 
@@ -116,6 +124,18 @@ __device__ inline bool mbar_test(uint32_t bar, uint32_t parity) {
       "selp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Blocking form: the thread is suspended until the phase completes or a time limit (at most
+// about `ns` nanoseconds) passes, so a waiting warp does not occupy issue slots.
+__device__ inline bool mbar_try(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
       : "memory");
   return ok != 0;
 }
@@ -202,25 +222,28 @@ __device__ inline void tmem_ld_wait(float* v) {
       :
       : "memory");
 }
-__device__ inline void named_barrier(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-// Barrier that also ORs a predicate over the participants: every thread gets the same answer,
-// so "stop now" decisions taken after it are uniform.
-__device__ inline bool named_barrier_or(int id, int count, bool pred) {
-  uint32_t r;
-  asm volatile(
-      "{\n.reg .pred p, q;\nsetp.ne.b32 q, %3, 0;\nbar.red.or.pred p, %1, %2, q;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(r)
-      : "r"(id), "r"(count), "r"((uint32_t)pred)
-      : "memory");
-  return r != 0;
-}
 __device__ inline float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ inline float fast_log2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// log2(2^a + 2^b) for values that may be -inf
+__device__ inline float lse2(float a, float b) {
+  const float hi = fmaxf(a, b), lo = fminf(a, b);
+  if (lo == -INFINITY) return hi;
+  return hi + fast_log2(1.0f + fast_exp2(lo - hi));
+}
+// counter increment that publishes this thread's earlier writes (and those ordered before it by
+// a barrier) and makes the writes of earlier incrementers visible to the caller
+__device__ inline int atom_add_acq_rel(int* p, int v) {
+  int old;
+  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
 }
 __device__ inline int ld_acquire(const int* p) {
   int v;
@@ -260,12 +283,12 @@ __device__ inline void give_up(Misc* m, unsigned* status) {
 // the drain waits at exit must outlast an abort to let copies in flight land).
 __device__ inline bool wait_bar(uint32_t bar, uint32_t parity, Misc* m, unsigned* status,
                                 bool heed_abort = true) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if (it > 64) {
-      if (heed_abort && m->abort_flag) return false;
-      __nanosleep(32);
-    }
+  if (mbar_try(bar, parity, 1000)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try(bar, parity, 1000)) return true;
+    if (heed_abort && m->abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) break;
   }
   give_up(m, status);
   return false;
@@ -390,12 +413,14 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       mbar_init(smem_u32(&m->s1_empty[s]), 128);
       mbar_init(smem_u32(&m->s2_full[s]), 1);
       mbar_init(smem_u32(&m->s2_empty[s]), 128);
-      mbar_init(smem_u32(&m->pub_full[s]), 128);
+      mbar_init(smem_u32(&m->pub_full[s]), 256);
       mbar_init(smem_u32(&m->pub_empty[s]), 1);
       mbar_init(smem_u32(&m->prep_full[s]), 1);
-      mbar_init(smem_u32(&m->prep_empty[s]), 1);
+      mbar_init(smem_u32(&m->prep_empty[s]), 2);
+      mbar_init(smem_u32(&m->gsync[s]), 128);
     }
     mbar_init(smem_u32(&m->drain), 1);
+    mbar_init(smem_u32(&m->drain2), 1);
     m->abort_flag = 0;
     m->p2_pos = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -420,10 +445,10 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         // stay within lag_keys of the score warps so pass 2 still finds its tiles in L2
         {
           const long long pos = key_pos(p, ck.head, (long long)ck.tile0 * kTile);
-          uint32_t spins = 0;
+          const long long t0 = clock64();
           while (pos > m->p2_pos + p.lag_keys && !m->abort_flag) {
-            __nanosleep(128);
-            if (++spins > kSpinLimit) give_up(m, p.status);
+            __nanosleep(200);
+            if (clock64() - t0 > kWaitCycles) give_up(m, p.status);
           }
           if (m->abort_flag) break;
         }
@@ -469,13 +494,14 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       // wait until the head's log-sum-exp and value norm are final
       bool ok = true;
       if (lane == 0) {
-        const int want_v = p.vbar_in ? 0 : kVWarps * ceil_div(ceil_div(ck.s.n, kTile), p.chunk_tiles);
-        uint32_t spins = 0;
+        const int want_v =
+            p.vbar_in ? 0 : kVWarps * ceil_div(ceil_div(ck.s.n, kTile), p.chunk_tiles);
+        const long long t0 = clock64();
         while (ld_acquire(&p.ready[ck.head]) == 0 ||
                (want_v && ld_acquire(&p.vcount[ck.head]) < want_v)) {
           if (m->abort_flag) break;
-          __nanosleep(64);
-          if (++spins > kSpinLimit) give_up(m, p.status);
+          __nanosleep(100);
+          if (clock64() - t0 > kWaitCycles) give_up(m, p.status);
         }
         ok = !m->abort_flag &&
              wait_bar(smem_u32(&m->prep_empty[slot]), (uint32_t)((j >> 1) & 1) ^ 1, m, p.status);
@@ -526,86 +552,53 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       if (q_loads > 0)
         wait_bar(smem_u32(&m->q2_full), (uint32_t)((q_loads - 1) & 1), m, p.status, false);
     }
-  } else if (warp == 2) {
-    // ================= MMA issuer: serves both pipelines by polling =========================
+  } else if (warp == 2 || warp == kMma2Warp) {
+    // ================= MMA issuers: warp 2 serves pass 1, the last warp pass 2 ================
     if (lane == 0) {
-      long long c1 = blockIdx.x, c2 = blockIdx.x;
-      long long n1 = 0, n2 = 0;
-      int t1 = 0, t2 = 0, nt1 = 0, nt2 = 0, q1_uses = 0, q2_uses = 0;
-      if (c1 < total1) nt1 = decode_chunk(p, m, c1, 1).ntiles;
-      if (c2 < total2) nt2 = decode_chunk(p, m, c2, 2).ntiles;
-      uint32_t idle = 0;
-      while (c1 < total1 || c2 < total2) {
-        bool progressed = false;
-        if (c1 < total1) {
-          const int st = (int)(n1 % kStages), buf = (int)(n1 & 1);
-          const bool need_q = t1 == 0;
-          if (mbar_test(smem_u32(&m->k1_full[st]), (uint32_t)((n1 / kStages) & 1)) &&
-              mbar_test(smem_u32(&m->s1_empty[buf]), (uint32_t)((n1 >> 1) & 1) ^ 1) &&
-              (!need_q || mbar_test(smem_u32(&m->q1_full), (uint32_t)(q1_uses & 1)))) {
-            if (need_q) ++q1_uses;
-            tc_fence_after();
-            const uint32_t d = tmem + (uint32_t)buf * 128u;
+      const bool first = warp == 2;
+      const int pass = first ? 1 : 2;
+      const long long total = first ? total1 : total2;
+      unsigned long long* k_full = first ? m->k1_full : m->k2_full;
+      unsigned long long* k_empty = first ? m->k1_empty : m->k2_empty;
+      unsigned long long* s_full = first ? m->s1_full : m->s2_full;
+      unsigned long long* s_empty = first ? m->s1_empty : m->s2_empty;
+      const uint32_t q_full = smem_u32(first ? &m->q1_full : &m->q2_full);
+      const uint32_t q_empty = smem_u32(first ? &m->q1_empty : &m->q2_empty);
+      const uint32_t q_addr = base + (first ? kOffQ1 : kOffQ2);
+      const uint32_t k_addr = base + (first ? kOffK1 : kOffK2);
+      const uint32_t d_base = tmem + (first ? 0u : 256u);
+      long long n = 0;
+      int q_uses = 0;
+      bool ok = true;
+      for (long long c = blockIdx.x; c < total && ok; c += gridDim.x) {
+        const int nt = decode_chunk(p, m, c, pass).ntiles;
+        ok = wait_bar(q_full, (uint32_t)(q_uses & 1), m, p.status);
+        ++q_uses;
+        for (int t = 0; t < nt && ok; ++t, ++n) {
+          const int st = (int)(n % kStages), buf = (int)(n & 1);
+          ok = wait_bar(smem_u32(&k_full[st]), (uint32_t)((n / kStages) & 1), m, p.status) &&
+               wait_bar(smem_u32(&s_empty[buf]), (uint32_t)((n >> 1) & 1) ^ 1, m, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d = d_base + (uint32_t)buf * 128u;
+          const uint32_t kt = k_addr + st * kTileBytes;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-              umma_bf16(d, make_desc(base + kOffQ1 + off),
-                        make_desc(base + kOffK1 + st * kTileBytes + off), kIdesc, kk > 0);
-            }
-            umma_commit(smem_u32(&m->k1_empty[st]));
-            umma_commit(smem_u32(&m->s1_full[buf]));
-            ++n1;
-            if (++t1 == nt1) {
-              // the query tile may be replaced once the MMAs of its last user have completed
-              umma_commit(smem_u32(&m->q1_empty));
-              t1 = 0;
-              c1 += gridDim.x;
-              if (c1 < total1) nt1 = decode_chunk(p, m, c1, 1).ntiles;
-            }
-            progressed = true;
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+            // pass 1: D[query, key] = Q K^T; pass 2: D[key, query] = K Q^T
+            if (first) umma_bf16(d, make_desc(q_addr + off), make_desc(kt + off), kIdesc, kk > 0);
+            else umma_bf16(d, make_desc(kt + off), make_desc(q_addr + off), kIdesc, kk > 0);
           }
+          umma_commit(smem_u32(&k_empty[st]));
+          umma_commit(smem_u32(&s_full[buf]));
         }
-        if (c2 < total2) {
-          const int st = (int)(n2 % kStages), buf = (int)(n2 & 1);
-          const bool need_q = t2 == 0;
-          if (mbar_test(smem_u32(&m->k2_full[st]), (uint32_t)((n2 / kStages) & 1)) &&
-              mbar_test(smem_u32(&m->s2_empty[buf]), (uint32_t)((n2 >> 1) & 1) ^ 1) &&
-              (!need_q || mbar_test(smem_u32(&m->q2_full), (uint32_t)(q2_uses & 1)))) {
-            if (need_q) ++q2_uses;
-            tc_fence_after();
-            const uint32_t d = tmem + 256u + (uint32_t)buf * 128u;
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-              umma_bf16(d, make_desc(base + kOffK2 + st * kTileBytes + off),
-                        make_desc(base + kOffQ2 + off), kIdesc, kk > 0);
-            }
-            umma_commit(smem_u32(&m->k2_empty[st]));
-            umma_commit(smem_u32(&m->s2_full[buf]));
-            ++n2;
-            if (++t2 == nt2) {
-              umma_commit(smem_u32(&m->q2_empty));
-              t2 = 0;
-              c2 += gridDim.x;
-              if (c2 < total2) nt2 = decode_chunk(p, m, c2, 2).ntiles;
-            }
-            progressed = true;
-          }
-        }
-        if (progressed) {
-          idle = 0;
-        } else if (++idle > 64) {
-          if (m->abort_flag) break;
-          __nanosleep(32);
-          if (idle > kSpinLimit) {
-            give_up(m, p.status);
-            break;
-          }
-        }
+        // the query tile may be replaced once the MMAs of its last user have completed
+        if (ok) umma_commit(q_empty);
       }
-      // every MMA has completed before TMEM is released
-      umma_commit(smem_u32(&m->drain));
-      wait_bar(smem_u32(&m->drain), 0, m, p.status, false);
+      // every MMA this thread issued has completed before TMEM is released
+      unsigned long long* drain = first ? &m->drain : &m->drain2;
+      umma_commit(smem_u32(drain));
+      wait_bar(smem_u32(drain), 0, m, p.status, false);
     }
   } else if (warp == 3) {
     // ================= publisher: chunk statistics leave the CTA; head folding ===============
@@ -618,80 +611,324 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         ok = wait_bar(smem_u32(&m->pub_full[slot]), (uint32_t)((j >> 1) & 1), m, p.status);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
-      float2* dst = p.part + ((size_t)ck.head * p.cph1_max + ck.index) * 128;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) dst[lane + 32 * q] = m->pub[slot][lane + 32 * q];
-      __threadfence();
+      // lane l carries rows 4l .. 4l+3; the two consumer groups' partials are merged first
+      {
+        const float4 a4 = reinterpret_cast<const float4*>(m->pub[slot][0])[lane];
+        const float4 b4 = reinterpret_cast<const float4*>(m->pub[slot][1])[lane];
+        float4 o4;
+        o4.x = lse2(a4.x, b4.x);
+        o4.y = lse2(a4.y, b4.y);
+        o4.z = lse2(a4.z, b4.z);
+        o4.w = lse2(a4.w, b4.w);
+        float* dst = p.part + ((size_t)ck.head * p.cph1_max + ck.index) * 128;
+        reinterpret_cast<float4*>(dst)[lane] = o4;
+      }
       __syncwarp();
       int last = 0;
       if (lane == 0) {
         mbar_arrive(smem_u32(&m->pub_empty[slot]));
-        last = atomicAdd(&p.counters[ck.head], 1) == ck.cph - 1;
+        last = atom_add_acq_rel(&p.counters[ck.head], 1) == ck.cph - 1;
       }
       last = __shfl_sync(0xffffffffu, last, 0);
       if (last) {
-        __threadfence();
         // fold the head's chunk partials, in chunk order, into one log-sum-exp per window query
-        const float2* pp = p.part + (size_t)ck.head * p.cph1_max * 128 + lane;
+        const float4* pp =
+            reinterpret_cast<const float4*>(p.part + (size_t)ck.head * p.cph1_max * 128) + lane;
         float big[4], sum[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           big[q] = -INFINITY;
           sum[q] = 0.f;
         }
-        for (int i0 = 0; i0 < ck.cph; i0 += 8) {
-          float2 pr[8][4];
+#pragma unroll 1
+        for (int i0 = 0; i0 < ck.cph; i0 += 16) {
+          float4 pr[16];
 #pragma unroll
-          for (int u = 0; u < 8; ++u)
+          for (int u = 0; u < 16; ++u)
+            pr[u] = (i0 + u < ck.cph) ? __ldcg(pp + (size_t)(i0 + u) * 32)
+                                      : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-              pr[u][q] = (i0 + u < ck.cph) ? __ldcg(pp + (size_t)(i0 + u) * 128 + 32 * q)
-                                           : make_float2(-INFINITY, 0.f);
+          for (int q = 0; q < 4; ++q) {
+            float l[16];
 #pragma unroll
-          for (int u = 0; u < 8; ++u)
+            for (int u = 0; u < 16; ++u)
+              l[u] = q == 0 ? pr[u].x : q == 1 ? pr[u].y : q == 2 ? pr[u].z : pr[u].w;
+            float bm = l[0];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float2 v = pr[u][q];
-              if (v.y > 0.f) {
-                if (v.x > big[q]) {
-                  sum[q] = sum[q] * fast_exp2(big[q] - v.x) + v.y;
-                  big[q] = v.x;
-                } else {
-                  sum[q] += v.y * fast_exp2(v.x - big[q]);
-                }
-              }
-            }
+            for (int u = 1; u < 16; ++u) bm = fmaxf(bm, l[u]);
+            const float nb = fmaxf(big[q], bm);
+            const float ref = nb == -INFINITY ? 0.f : nb;  // keeps -inf - -inf out of the exponent
+            float acc = sum[q] * fast_exp2(big[q] - ref);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) acc += fast_exp2(l[u] - ref);
+            sum[q] = acc;
+            big[q] = nb;
+          }
         }
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          p.neg_lse[(size_t)ck.head * 128 + lane + 32 * q] =
-              sum[q] > 0.f ? -(big[q] + log2f(sum[q])) : -INFINITY;
-        __threadfence();
+        float4 out;
+        out.x = sum[0] > 0.f ? -(big[0] + fast_log2(sum[0])) : -INFINITY;
+        out.y = sum[1] > 0.f ? -(big[1] + fast_log2(sum[1])) : -INFINITY;
+        out.z = sum[2] > 0.f ? -(big[2] + fast_log2(sum[2])) : -INFINITY;
+        out.w = sum[3] > 0.f ? -(big[3] + fast_log2(sum[3])) : -INFINITY;
+        reinterpret_cast<float4*>(p.neg_lse + (size_t)ck.head * 128)[lane] = out;
         __syncwarp();
         if (lane == 0) st_release(&p.ready[ck.head], 1);
       }
     }
-  } else if (warp >= 4 && warp < 8) {
-    // ================= pass-1 consumers: one thread per (query head, window query) row ======
-    const int quad = warp & 3, row = quad * 32 + lane;
+  } else if (warp >= 4 && warp < 12) {
+    // ================= consumers: two groups of four warps, each serving BOTH passes ==========
+    // Group 0 owns TMEM buffer 0 of either pipeline (the even tiles a CTA sees), group 1 buffer
+    // 1.  A group takes whichever of its tiles is ready, pass 2 first, so the exponential unit
+    // of every scheduler always has two warps to draw from while either pass has work.
+    //   pass 1: thread = (query head, window query) row, running (max, sum of exp2) per chunk
+    //   pass 2: thread = key, window-mean attention per query head, pooling, score, entropy
+    constexpr int NH = 128 / W;  // query heads that fit the 128 columns
+    const int grp = (warp - 4) >> 2, quad = warp & 3, row = quad * 32 + lane;
     const int t_in_win = row % W;
+    const int rad = g.pool_radius;
+    const float inv_w = 1.0f / (float)W;
     const float sc2 = g.scale_log2;
-    long long n = 0, j = 0;
+    const bool avg = g.pool_kind == LAVA_POOL_AVG;
+    const uint32_t gbar = smem_u32(&m->gsync[grp]);
+    uint32_t gphase = 0;
     bool alive = true;
-    for (long long c = blockIdx.x; c < total1 && alive; c += gridDim.x, ++j) {
-      const Chunk ck = decode_chunk(p, m, c, 1);
+    // rendezvous of the group's four warps (bounded, and it ends when the CTA aborts)
+    auto group_sync = [&]() {
+      mbar_arrive(gbar);
+      if (!__all_sync(0xffffffffu, wait_bar(gbar, gphase & 1, m, p.status))) alive = false;
+      ++gphase;
+    };
+
+    // ---- cursors over the CTA's chunks of both passes ---------------------------------------
+    long long c1 = blockIdx.x, n1 = 0, j1 = 0;
+    int t1 = 0, last1 = 0;
+    bool has1 = c1 < total1;
+    Chunk k1;
+    float mx = -INFINITY, z = 0.f;
+    auto open1 = [&]() {
+      k1 = decode_chunk(p, m, c1, 1);
       // keys this query may see: i < n and i <= P + t
-      const int last = row < rows_valid ? min(ck.s.n, ck.s.prefix + t_in_win + 1) : 0;
-      float mx = -INFINITY, z = 0.f;
-      for (int t = 0; t < ck.ntiles; ++t, ++n) {
-        const int buf = (int)(n & 1);
-        alive = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->s1_full[buf]),
-                                                 (uint32_t)((n >> 1) & 1), m, p.status));
-        if (!alive) break;
+      last1 = row < rows_valid ? min(k1.s.n, k1.s.prefix + t_in_win + 1) : 0;
+    };
+    if (has1) open1();
+    long long c2 = blockIdx.x, n2 = 0, j2 = 0;
+    int t2 = 0;
+    bool has2 = c2 < total2, prepped = false;
+    Chunk k2;
+    float es = 0.f, et = 0.f;  // entropy sums of this thread's keys over the chunk
+    if (has2) k2 = decode_chunk(p, m, c2, 2);
+    if (grp == 0 && row == 0 && has2)
+      m->p2_pos = key_pos(p, k2.head, (long long)k2.tile0 * p.out_keys);
+
+    uint32_t idle = 0;
+    long long idle_t0 = 0;
+    while (alive) {
+      // ---- move the pass-1 cursor to this group's next tile; close finished chunks ----------
+      while (has1 && alive) {
+        if (t1 == k1.ntiles) {
+          // hand the chunk's statistics (as one log2-sum-exp) to the publisher warp
+          const int slot = (int)(j1 & 1);
+          if (!__all_sync(0xffffffffu, wait_bar(smem_u32(&m->pub_empty[slot]),
+                                                (uint32_t)((j1 >> 1) & 1) ^ 1, m, p.status))) {
+            alive = false;
+            break;
+          }
+          m->pub[slot][grp][row] = z > 0.f ? mx + fast_log2(z) : -INFINITY;
+          mbar_arrive(smem_u32(&m->pub_full[slot]));
+          mx = -INFINITY;
+          z = 0.f;
+          ++j1;
+          c1 += gridDim.x;
+          t1 = 0;
+          has1 = c1 < total1;
+          if (has1) open1();
+          continue;
+        }
+        if ((int)(n1 & 1) == grp) break;
+        ++t1;  // the other group's tile
+        ++n1;
+      }
+      // ---- the same for pass 2 ----------------------------------------------------------------
+      while (has2 && alive) {
+        if (t2 == k2.ntiles) {
+          // entropy sums of the chunk in a fixed order: keys of a thread, lanes, then warps
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            es += __shfl_down_sync(0xffffffffu, es, o);
+            et += __shfl_down_sync(0xffffffffu, et, o);
+          }
+          if (lane == 0) {
+            m->red[grp][0][quad] = es;
+            m->red[grp][1][quad] = et;
+          }
+          group_sync();
+          if (!alive) break;
+          if (row == 0) {
+            const float(*r)[4] = m->red[grp];
+            const double s_sum = ((double)r[0][0] + (double)r[0][1]) + ((double)r[0][2] + (double)r[0][3]);
+            const double t_sum = ((double)r[1][0] + (double)r[1][1]) + ((double)r[1][2] + (double)r[1][3]);
+            p.ent_part[((size_t)k2.head * p.cph2_max + k2.index) * 2 + grp] = make_double2(s_sum, t_sum);
+            mbar_arrive(smem_u32(&m->prep_empty[j2 & 1]));
+            if (grp == 0) {
+              // the throttle of pass 1 follows the first key this CTA has still to score
+              long long next = 0x3fffffffffffffffLL;
+              if (c2 + gridDim.x < total2) {
+                const Chunk nx = decode_chunk(p, m, c2 + gridDim.x, 2);
+                next = key_pos(p, nx.head, (long long)nx.tile0 * p.out_keys);
+              }
+              m->p2_pos = next;
+            }
+          }
+          group_sync();  // red[] is free again
+          if (!alive) break;
+          es = 0.f;
+          et = 0.f;
+          prepped = false;
+          ++j2;
+          c2 += gridDim.x;
+          t2 = 0;
+          has2 = c2 < total2;
+          if (has2) k2 = decode_chunk(p, m, c2, 2);
+          continue;
+        }
+        if ((int)(n2 & 1) == grp) break;
+        ++t2;
+        ++n2;
+      }
+      if (!alive || (!has1 && !has2)) break;
+
+      bool did = false;
+      // ---- a pass-2 tile: scores of 128 - 2 * pool_radius keys ----------------------------------
+      if (has2) {
+        if (!prepped)
+          prepped = __all_sync(0xffffffffu, mbar_test(smem_u32(&m->prep_full[j2 & 1]),
+                                                      (uint32_t)((j2 >> 1) & 1)));
+        if (prepped && __all_sync(0xffffffffu, mbar_test(smem_u32(&m->s2_full[grp]),
+                                                         (uint32_t)((n2 >> 1) & 1)))) {
+          did = true;
+          const Prep* prep = &m->prep[j2 & 1];
+          const int tile = k2.tile0 + t2;
+          tc_fence_after();
+          float acc[NH];
+#pragma unroll
+          for (int h = 0; h < NH; ++h) acc[h] = 0.f;
+          const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)grp * 128u;
+          // window queries come in blocks of 32 columns; a block lies inside one query head
+          // when W >= 32, and holds two heads when W == 16
+          const int nblk = (rows_valid + 31) >> 5;
+#pragma unroll 1
+          for (int blk = 0; blk < nblk; ++blk) {
+            float cur[32], l[32];
+            tmem_ld32_issue(taddr + blk * 32, cur);
+            // the block's log-sum-exp values travel to registers while the TMEM load is in flight
+#pragma unroll
+            for (int c4 = 0; c4 < 32; c4 += 4) {
+              const float4 l4 = *reinterpret_cast<const float4*>(&prep->lse[blk * 32 + c4]);
+              l[c4 + 0] = l4.x;
+              l[c4 + 1] = l4.y;
+              l[c4 + 2] = l4.z;
+              l[c4 + 3] = l4.w;
+            }
+            tmem_ld_wait(cur);
+            // stage by stage, so that independent operations follow one another in issue order
+#pragma unroll
+            for (int i = 0; i < 32; ++i) cur[i] = fmaf(cur[i], sc2, l[i]);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i]);
+            if (W >= 32) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) cur[i] += cur[i + 16];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) cur[i] += cur[i + 8];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) cur[i] += cur[i + 4];
+              const float sum = (cur[0] + cur[1]) + (cur[2] + cur[3]);
+              const int h = (blk * 32) / W;
+#pragma unroll
+              for (int hh = 0; hh < NH; ++hh)
+                if (hh == h) acc[hh] += sum;
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                cur[i] += cur[i + 8];
+                cur[16 + i] += cur[24 + i];
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                cur[i] += cur[i + 4];
+                cur[16 + i] += cur[20 + i];
+              }
+              const float s0 = (cur[0] + cur[1]) + (cur[2] + cur[3]);
+              const float s1 = (cur[16] + cur[17]) + (cur[18] + cur[19]);
+#pragma unroll
+              for (int hh = 0; hh < NH; hh += 2)
+                if (hh == 2 * blk) {
+                  acc[hh] += s0;
+                  if (hh + 1 < NH) acc[hh + 1] += s1;
+                }
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(smem_u32(&m->s2_empty[grp]));
+          // lane <-> key: the tile starts pool_radius keys before the first key it owns; keys
+          // outside the prefix hold the neutral element of both pools (values are >= 0)
+          const int ab = (int)((n2 >> 1) & 1);
+          const int key0 = tile * p.out_keys - rad;
+          const int i = key0 + row;
+          const bool inside = i >= 0 && i < k2.s.prefix;
+          float(*abuf)[kTile] = m->a[grp][ab];
+          if (avg) {
+#pragma unroll
+            for (int h = 0; h < NH; ++h) abuf[h][row] = inside ? acc[h] * inv_w : 0.f;
+          } else {
+            // max-pooling commutes with the group maximum: reduce over the query heads first
+            float top = 0.f;
+#pragma unroll
+            for (int h = 0; h < NH; ++h)
+              if (h < g.group) top = fmaxf(top, acc[h] * inv_w);
+            abuf[0][row] = inside ? top : 0.f;
+          }
+          group_sync();
+          if (!alive) break;
+          const int own_lo = tile * p.out_keys, own_hi = min(k2.s.prefix, own_lo + p.out_keys);
+          if (i >= own_lo && i < own_hi) {
+            float best = 0.f;
+            if (avg) {
+              for (int h = 0; h < g.group; ++h) {
+                const float* a = &abuf[h][row];
+                float pv = 0.f;
+                for (int q = -rad; q <= rad; ++q) pv += a[q];
+                best = fmaxf(best, pv / (float)g.pool_kernel);
+              }
+            } else {
+              const float* a = &abuf[0][row];
+              if (rad == 3) {
+                best = fmaxf(fmaxf(fmaxf(a[-3], a[-2]), fmaxf(a[-1], a[0])),
+                             fmaxf(fmaxf(a[1], a[2]), a[3]));
+              } else {
+                best = a[0];
+                for (int q = 1; q <= rad; ++q) best = fmaxf(best, fmaxf(a[-q], a[q]));
+              }
+            }
+            const float sc = best * prep->scale;
+            p.scores[(size_t)k2.layer * g.total_scores + k2.s.score_off +
+                     (long long)k2.kvh * k2.s.prefix + i] = sc;
+            if (sc > 0.f) {
+              es += sc;
+              et += sc * __logf(sc);
+            }
+          }
+          ++t2;
+          ++n2;
+        }
+      }
+      // ---- a pass-1 tile: running softmax statistics of 128 keys --------------------------------
+      if (!did && has1 &&
+          __all_sync(0xffffffffu, mbar_test(smem_u32(&m->s1_full[grp]), (uint32_t)((n1 >> 1) & 1)))) {
+        did = true;
         tc_fence_after();
-        const int limit = max(0, min(kTile, last - (ck.tile0 + t) * kTile));
-        const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * 128u;
-        // a compact loop body: the four warp roles of a scheduler share its instruction cache
+        const int limit = max(0, min(kTile, last1 - (k1.tile0 + t1) * kTile));
+        const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)grp * 128u;
 #pragma unroll 1
         for (int blk = 0; blk < 4; ++blk) {
           const int cnt = limit - blk * 32;
@@ -699,26 +936,31 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           tmem_ld32_issue(taddr + blk * 32, cur);
           tmem_ld_wait(cur);
           if (cnt >= 32) {
-            float b0 = fmaxf(cur[0], cur[1]), b1 = fmaxf(cur[2], cur[3]);
+            // stage by stage (maxima, scaled differences, exponentials, a fixed summation tree)
+            float t[16];
 #pragma unroll
-            for (int i = 4; i < 32; i += 4) {
-              b0 = fmaxf(b0, fmaxf(cur[i], cur[i + 1]));
-              b1 = fmaxf(b1, fmaxf(cur[i + 2], cur[i + 3]));
-            }
-            const float nm = fmaxf(b0, b1) * sc2;
+            for (int i = 0; i < 16; ++i) t[i] = fmaxf(cur[i], cur[i + 16]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t[i] = fmaxf(t[i], t[i + 8]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t[i] = fmaxf(t[i], t[i + 4]);
+            const float nm = fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3])) * sc2;
             if (nm > mx) {
               z *= fast_exp2(mx - nm);
               mx = nm;
             }
-            float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+            const float neg = -mx;
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              z0 += fast_exp2(fmaf(cur[i + 0], sc2, -mx));
-              z1 += fast_exp2(fmaf(cur[i + 1], sc2, -mx));
-              z2 += fast_exp2(fmaf(cur[i + 2], sc2, -mx));
-              z3 += fast_exp2(fmaf(cur[i + 3], sc2, -mx));
-            }
-            z += (z0 + z1) + (z2 + z3);
+            for (int i = 0; i < 32; ++i) cur[i] = fmaf(cur[i], sc2, neg);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i]);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) cur[i] += cur[i + 16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cur[i] += cur[i + 8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cur[i] += cur[i + 4];
+            z += (cur[0] + cur[1]) + (cur[2] + cur[3]);
           } else if (cnt > 0) {
             float bm = -INFINITY;
 #pragma unroll
@@ -737,186 +979,31 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           }
         }
         tc_fence_before();
-        mbar_arrive(smem_u32(&m->s1_empty[buf]));
+        mbar_arrive(smem_u32(&m->s1_empty[grp]));
+        ++t1;
+        ++n1;
       }
-      if (!alive) break;
-      // hand the chunk's statistics to the publisher warp
-      const int slot = (int)(j & 1);
-      alive = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->pub_empty[slot]),
-                                               (uint32_t)((j >> 1) & 1) ^ 1, m, p.status));
-      if (!alive) break;
-      m->pub[slot][row] = make_float2(mx, z);
-      mbar_arrive(smem_u32(&m->pub_full[slot]));
-    }
-  } else if (warp >= 8 && warp < 12) {
-    // ================= pass-2 consumers: one thread per key ==================================
-    constexpr int NH = 128 / W;  // query heads that fit the 128 columns
-    const int quad = warp & 3, key_lane = quad * 32 + lane, tid = key_lane;
-    const int rad = g.pool_radius;
-    const float inv_w = 1.0f / (float)W;
-    const float sc2 = g.scale_log2;
-    long long n = 0, j = 0;
-    bool alive = true;
-    if (tid == 0 && (long long)blockIdx.x < total2) {
-      const Chunk first = decode_chunk(p, m, blockIdx.x, 2);
-      m->p2_pos = key_pos(p, first.head, (long long)first.tile0 * p.out_keys);
-    }
-    // Exits are taken only after a barrier that ORs the stop condition over all four warps, so
-    // no warp is ever left waiting at a barrier the others have abandoned.
-    for (long long c = blockIdx.x; c < total2 && alive; c += gridDim.x, ++j) {
-      const Chunk ck = decode_chunk(p, m, c, 2);
-      const int slot = (int)(j & 1);
-      const bool got = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->prep_full[slot]),
-                                                        (uint32_t)((j >> 1) & 1), m, p.status));
-      if (named_barrier_or(2, 128, !got || m->abort_flag != 0)) break;
-      const Prep* prep = &m->prep[slot];
-      const float head_scale = prep->scale;
-      float es = 0.f, et = 0.f;  // entropy sums of this thread's keys over the chunk
-      for (int t = 0; t < ck.ntiles; ++t, ++n) {
-        const int tile = ck.tile0 + t;
-        const int buf = (int)(n & 1);
-        const bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&m->s2_full[buf]),
-                                                         (uint32_t)((n >> 1) & 1), m, p.status));
-        tc_fence_after();
-        float acc[NH];
-#pragma unroll
-        for (int h = 0; h < NH; ++h) acc[h] = 0.f;
-        if (ok) {  // warp-uniform: the TMEM loads below are executed by whole warps
-          const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)buf * 128u;
-          // window queries come in blocks of 32 columns; a block never straddles two query
-          // heads when W >= 32, and covers 32 / W whole heads otherwise
-          const int nblk = (rows_valid + 31) >> 5;
-#pragma unroll 1
-          for (int blk = 0; blk < nblk; ++blk) {
-            float cur[32];
-            tmem_ld32_issue(taddr + blk * 32, cur);
-            tmem_ld_wait(cur);
-            const float* lse = &prep->lse[blk * 32];
-            if (W >= 32) {
-              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-              for (int c4 = 0; c4 < 32; c4 += 4) {
-                const float4 l4 = *reinterpret_cast<const float4*>(lse + c4);
-                s0 += fast_exp2(fmaf(cur[c4 + 0], sc2, l4.x));
-                s1 += fast_exp2(fmaf(cur[c4 + 1], sc2, l4.y));
-                s2 += fast_exp2(fmaf(cur[c4 + 2], sc2, l4.z));
-                s3 += fast_exp2(fmaf(cur[c4 + 3], sc2, l4.w));
-              }
-              const float sum = (s0 + s1) + (s2 + s3);
-              const int h = (blk * 32) / W;
-#pragma unroll
-              for (int hh = 0; hh < NH; ++hh)
-                if (hh == h) acc[hh] += sum;
-            } else {  // W == 16: two query heads per block
-              float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-              for (int c4 = 0; c4 < 16; c4 += 4) {
-                const float4 l4 = *reinterpret_cast<const float4*>(lse + c4);
-                const float4 r4 = *reinterpret_cast<const float4*>(lse + 16 + c4);
-                s0 += (fast_exp2(fmaf(cur[c4 + 0], sc2, l4.x)) + fast_exp2(fmaf(cur[c4 + 1], sc2, l4.y))) +
-                      (fast_exp2(fmaf(cur[c4 + 2], sc2, l4.z)) + fast_exp2(fmaf(cur[c4 + 3], sc2, l4.w)));
-                s1 += (fast_exp2(fmaf(cur[16 + c4 + 0], sc2, r4.x)) + fast_exp2(fmaf(cur[16 + c4 + 1], sc2, r4.y))) +
-                      (fast_exp2(fmaf(cur[16 + c4 + 2], sc2, r4.z)) + fast_exp2(fmaf(cur[16 + c4 + 3], sc2, r4.w)));
-              }
-#pragma unroll
-              for (int hh = 0; hh < NH; hh += 2)
-                if (hh == 2 * blk) {
-                  acc[hh] += s0;
-                  if (hh + 1 < NH) acc[hh + 1] += s1;
-                }
-            }
-          }
-          tc_fence_before();
-          mbar_arrive(smem_u32(&m->s2_empty[buf]));
-        }
-        // lane <-> key: the tile starts pool_radius keys before the first key it owns; keys
-        // outside the prefix hold the neutral element of both pools (values are >= 0)
-        const int ab = (int)(n & 1);
-        const int key0 = tile * p.out_keys - rad;
-        const int i = key0 + key_lane;
-        const bool inside = i >= 0 && i < ck.s.prefix;
-        const bool avg = g.pool_kind == LAVA_POOL_AVG;
-        if (avg) {
-#pragma unroll
-          for (int h = 0; h < NH; ++h) m->a[ab][h][key_lane] = inside ? acc[h] * inv_w : 0.f;
-        } else {
-          // max-pooling commutes with the group maximum: reduce over the query heads first
-          float top = 0.f;
-#pragma unroll
-          for (int h = 0; h < NH; ++h)
-            if (h < g.group) top = fmaxf(top, acc[h] * inv_w);
-          m->a[ab][0][key_lane] = inside ? top : 0.f;
-        }
-        if (named_barrier_or(2, 128, !ok || m->abort_flag != 0)) {
-          alive = false;
+      if (did) {
+        idle = 0;
+      } else {
+        // nothing ready for this group: step aside for a moment (bounded)
+        if (idle++ == 0) idle_t0 = clock64();
+        if (m->abort_flag) break;
+        __nanosleep(kBackoffNs);
+        if (clock64() - idle_t0 > kWaitCycles) {
+          give_up(m, p.status);
           break;
         }
-        const int own_lo = tile * p.out_keys, own_hi = min(ck.s.prefix, own_lo + p.out_keys);
-        if (i >= own_lo && i < own_hi) {
-          float best = 0.f;
-          if (avg) {
-            for (int h = 0; h < g.group; ++h) {
-              const float* a = &m->a[ab][h][key_lane];
-              float pv = 0.f;
-              for (int q = -rad; q <= rad; ++q) pv += a[q];
-              best = fmaxf(best, pv / (float)g.pool_kernel);
-            }
-          } else {
-            const float* a = &m->a[ab][0][key_lane];
-            if (rad == 3) {
-              best = fmaxf(fmaxf(fmaxf(a[-3], a[-2]), fmaxf(a[-1], a[0])),
-                           fmaxf(fmaxf(a[1], a[2]), a[3]));
-            } else {
-              best = a[0];
-              for (int q = 1; q <= rad; ++q) best = fmaxf(best, fmaxf(a[-q], a[q]));
-            }
-          }
-          const float sc = best * head_scale;
-          p.scores[(size_t)ck.layer * g.total_scores + ck.s.score_off +
-                   (long long)ck.kvh * ck.s.prefix + i] = sc;
-          if (sc > 0.f) {
-            es += sc;
-            et += sc * __logf(sc);
-          }
-        }
       }
-      if (!alive) break;
-      // entropy sums of the chunk in a fixed order: keys of a thread, lanes, then warps
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        es += __shfl_down_sync(0xffffffffu, es, o);
-        et += __shfl_down_sync(0xffffffffu, et, o);
-      }
-      if (lane == 0) {
-        m->red[0][quad] = es;
-        m->red[1][quad] = et;
-      }
-      named_barrier(2, 128);
-      if (tid == 0) {
-        const double s_sum = ((double)m->red[0][0] + (double)m->red[0][1]) +
-                             ((double)m->red[0][2] + (double)m->red[0][3]);
-        const double t_sum = ((double)m->red[1][0] + (double)m->red[1][1]) +
-                             ((double)m->red[1][2] + (double)m->red[1][3]);
-        p.ent_part[(size_t)ck.head * p.cph2_max + ck.index] = make_double2(s_sum, t_sum);
-        mbar_arrive(smem_u32(&m->prep_empty[slot]));
-        // the throttle of pass 1 follows the first key this CTA has still to score
-        long long next = 0x3fffffffffffffffLL;
-        if (c + gridDim.x < total2) {
-          const Chunk nx = decode_chunk(p, m, c + gridDim.x, 2);
-          next = key_pos(p, nx.head, (long long)nx.tile0 * p.out_keys);
-        }
-        m->p2_pos = next;
-      }
-      named_barrier(2, 128);  // red[] is free again
     }
-    if (tid == 0) m->p2_pos = 0x3fffffffffffffffLL;  // pass 1 is no longer held back
-  } else {
+    if (grp == 0 && row == 0) m->p2_pos = 0x3fffffffffffffffLL;  // pass 1 is no longer held back
+  } else if (warp >= 12 && warp < 12 + kVWarps) {
     // ================= value-norm warps: the V rows of the CTA's pass-1 chunks ===============
-    // 256 threads, 16 per row.  Rows are taken in groups of 128 (8 loads of 16 B per thread);
+    // 224 threads, 16 per row.  Rows are taken in groups of 112 (8 loads of 16 B per thread);
     // one group is in flight while the previous one is reduced, across chunk borders too.
     if (!p.vbar_in) {
       const uint64_t drop = policy_evict_first();
-      const int vt = threadIdx.x - 12 * 32;       // 0..255
+      const int vt = threadIdx.x - 12 * 32;       // 0..223
       const int sub = vt >> 4, piece = vt & 15;
       struct Group {
         const char* base;  // this thread's 16 bytes of row 0 of the sequence
@@ -932,11 +1019,11 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           ck = decode_chunk(p, m, c, 1);
           c += gridDim.x;
           grp = 0;
-          ngrp = ceil_div(min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile) - ck.tile0 * kTile, 128);
+          ngrp = ceil_div(min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile) - ck.tile0 * kTile, 8 * kVRows);
         }
         gr.base = p.v + ((size_t)ck.layer * p.v_ls + (long long)ck.kvh * g.v_sh +
                          ck.s.tok0 * g.v_st) * 2 + piece * 16;
-        gr.row0 = ck.tile0 * kTile + grp * 128 + sub;
+        gr.row0 = ck.tile0 * kTile + grp * 8 * kVRows + sub;
         gr.row_hi = min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile);
         gr.head = ck.head;
         gr.last = ++grp == ngrp;
@@ -945,7 +1032,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       auto issue = [&](uint4 (&buf)[8], const Group& gr) {
 #pragma unroll
         for (int s8 = 0; s8 < 8; ++s8) {
-          const int row = gr.row0 + s8 * 16;
+          const int row = gr.row0 + s8 * kVRows;
           buf[s8] = make_uint4(0, 0, 0, 0);
           if (row < gr.row_hi) buf[s8] = ld_stream16(gr.base + (long long)row * g.v_st * 2, drop);
         }
@@ -1028,9 +1115,9 @@ entropy_finalize_sm100_kernel(Geom g, const double2* ent_part, int cph2_max, int
   double sum_s = 0.0, sum_t = 0.0;
   for (int i = threadIdx.x; i < total; i += 256) {
     const int kvh = i / used, t = i - kvh * used;
-    const double2 v = ent_part[((size_t)prob * g.n_kv_heads + kvh) * cph2_max + t];
-    sum_s += v.x;
-    sum_t += v.y;
+    const double2* e = ent_part + (((size_t)prob * g.n_kv_heads + kvh) * cph2_max + t) * 2;
+    sum_s += e[0].x + e[1].x;  // the two consumer groups of the chunk
+    sum_t += e[0].y + e[1].y;
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -1088,6 +1175,19 @@ int chunk_tiles_setting() {
   return value;
 }
 
+
+// rounds of chunks pass 1 may run ahead of a head's completion: tuning knob
+// (LAVA_SM100_LAG_ROUNDS), default 2
+int lag_rounds_setting() {
+  static int value = -1;
+  if (value < 0) {
+    const char* e = getenv("LAVA_SM100_LAG_ROUNDS");
+    const int v = e ? atoi(e) : -1;
+    value = (v >= 0 && v <= 4096) ? v : 2;
+  }
+  return value;
+}
+
 }  // namespace
 
 bool sm100_supported(const Geom& g) {
@@ -1111,11 +1211,11 @@ Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   off = up256(off + sizeof(int) * 4 * (size_t)l.heads_total);
   l.sync_bytes = off;
   l.off_part = off;
-  off = up256(off + sizeof(float2) * 128 * (size_t)l.heads_total * l.tiles1);
+  off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total * l.tiles1);
   l.off_lse = off;
   off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total);
   l.off_ent = off;
-  off = up256(off + sizeof(double2) * (size_t)l.heads_total * l.tiles2);
+  off = up256(off + sizeof(double2) * 2 * (size_t)l.heads_total * l.tiles2);
   l.total = off;
   return l;
 }
@@ -1171,7 +1271,7 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.cph2_max = lay.tiles2;
   // Pass 1 must be allowed to finish the head pass 2 is waiting for (one head = max_seqlen
   // keys); two further rounds of chunks cover the time the head's statistics take to fold.
-  p.lag_keys = (long long)g.max_seqlen + 2LL * sms * p.chunk_tiles * kTile;
+  p.lag_keys = (long long)g.max_seqlen + (long long)lag_rounds_setting() * sms * p.chunk_tiles * kTile;
   p.vbar_in = vbar_in;
   p.scores = scores;
   p.vbar_out = vbar_out;
@@ -1181,7 +1281,7 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.ready = p.counters + lay.heads_total;
   p.vcount = p.ready + lay.heads_total;
   p.vbar_bits = reinterpret_cast<unsigned*>(p.vcount + lay.heads_total);
-  p.part = reinterpret_cast<float2*>(ws + lay.off_part);
+  p.part = reinterpret_cast<float*>(ws + lay.off_part);
   p.neg_lse = reinterpret_cast<float*>(ws + lay.off_lse);
   p.ent_part = reinterpret_cast<double2*>(ws + lay.off_ent);
   p.status = reinterpret_cast<unsigned*>(ws_base);  // the status word opens the workspace
