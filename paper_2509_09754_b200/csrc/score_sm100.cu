@@ -43,7 +43,6 @@ constexpr int kMaxBatch = 512;       // sequences the in-kernel chunk schedule c
 constexpr uint32_t kTileBytes = 128 * 128 * 2;  // one [128 x 128] bf16 tile = 2 swizzled blocks
 constexpr uint32_t kHalfBytes = kTileBytes / 2;
 constexpr long long kWaitCycles = 1ll << 32;  // every wait gives up after about two seconds
-constexpr unsigned kBackoffNs = 40;           // pause of a consumer group that found no tile ready
 
 // shared memory map (bytes from a 1024-aligned base)
 constexpr uint32_t kOffQ1 = 0;
@@ -67,14 +66,12 @@ struct Misc {
   unsigned long long pub_full[2], pub_empty[2], prep_full[2], prep_empty[2];
   unsigned long long gsync[2];        // rendezvous of the four warps of a consumer group
   unsigned long long drain, drain2;
-  volatile long long p2_pos;  // first key (global key coordinate) pass 2 has not finished yet
   uint32_t tmem_base;
   volatile int abort_flag;
   int sched_total1, sched_total2;     // chunks per layer of pass 1 / pass 2
   alignas(16) float pub[2][2][128];   // [slot][group][query]: log2-sum-exp of a finished chunk
   Prep prep[2];
   alignas(16) float a[2][2][8][kTile];  // [group][tile parity][query head][key]: window means
-  float red[2][2][4];                 // [group][S or T][warp]
   int pref1[kMaxBatch + 1], pref2[kMaxBatch + 1];  // exclusive scans of chunks per sequence
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
@@ -85,7 +82,7 @@ struct Sm100Params {
   int chunk_tiles;          // tiles per chunk
   int out_keys;             // keys a pass-2 tile owns: 128 - 2 * pool_radius
   int cph1_max, cph2_max;   // chunks per head at max_seqlen (strides of the scratch arrays)
-  long long lag_keys;       // pass 1 may run this many keys ahead of pass 2
+  long long lag_keys;       // a pass-1 tile may start this many keys beyond the next pass-2 tile
   const float* vbar_in;
   float* scores;
   float* vbar_out;
@@ -98,7 +95,7 @@ struct Sm100Params {
   int* vcount;              // [heads_total] finished value-norm warps
   unsigned* vbar_bits;      // [heads_total]
   float* neg_lse;           // [heads_total][128]
-  double2* ent_part;        // [heads_total][cph2_max][2 consumer groups]
+  float2* ent_part;         // [heads_total][cph2_max][8 consumer warps] (sum s, sum s ln s)
   unsigned* status;
 };
 
@@ -116,16 +113,6 @@ __device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ inline void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ inline bool mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
 }
 // Blocking form: the thread is suspended until the phase completes or a time limit (at most
 // about `ns` nanoseconds) passes, so a waiting warp does not occupy issue slots.
@@ -310,12 +297,12 @@ __device__ inline int tiles_of(const Sm100Params& p, const SeqInfo& s, int pass)
   return pass == 1 ? ceil_div(s.n, kTile) : ceil_div(s.prefix, p.out_keys);
 }
 
-__device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, long long c, int pass) {
+__device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, int c, int pass) {
   const int* pref = pass == 1 ? m->pref1 : m->pref2;
   const int per_layer = pass == 1 ? m->sched_total1 : m->sched_total2;
   Chunk ck;
-  ck.layer = (int)(c / per_layer);
-  const int r = (int)(c - (long long)ck.layer * per_layer);
+  ck.layer = c / per_layer;
+  const int r = c - ck.layer * per_layer;
   const int hkv = p.g.n_kv_heads;
   int lo = 0, hi = p.g.batch;  // largest b with hkv * pref[b] <= r
   while (hi - lo > 1) {
@@ -334,7 +321,7 @@ __device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, long l
   return ck;
 }
 
-// global key coordinate used by the pass-1 throttle
+// global key coordinate that orders the tiles of the two passes
 __device__ inline long long key_pos(const Sm100Params& p, int head, long long key) {
   return (long long)head * p.g.max_seqlen + key;
 }
@@ -416,13 +403,12 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       mbar_init(smem_u32(&m->pub_full[s]), 256);
       mbar_init(smem_u32(&m->pub_empty[s]), 1);
       mbar_init(smem_u32(&m->prep_full[s]), 1);
-      mbar_init(smem_u32(&m->prep_empty[s]), 2);
+      mbar_init(smem_u32(&m->prep_empty[s]), 8);
       mbar_init(smem_u32(&m->gsync[s]), 128);
     }
     mbar_init(smem_u32(&m->drain), 1);
     mbar_init(smem_u32(&m->drain2), 1);
     m->abort_flag = 0;
-    m->p2_pos = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -442,16 +428,6 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       long long n = 0;  // K loads issued
       for (long long c = blockIdx.x; c < total1 && !m->abort_flag; c += gridDim.x) {
         const Chunk ck = decode_chunk(p, m, c, 1);
-        // stay within lag_keys of the score warps so pass 2 still finds its tiles in L2
-        {
-          const long long pos = key_pos(p, ck.head, (long long)ck.tile0 * kTile);
-          const long long t0 = clock64();
-          while (pos > m->p2_pos + p.lag_keys && !m->abort_flag) {
-            __nanosleep(200);
-            if (clock64() - t0 > kWaitCycles) give_up(m, p.status);
-          }
-          if (m->abort_flag) break;
-        }
         if (!wait_bar(smem_u32(&m->q1_empty), (q_loads & 1) ^ 1, m, p.status)) break;
         {
           const uint32_t bar = smem_u32(&m->q1_full);
@@ -678,10 +654,14 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
   } else if (warp >= 4 && warp < 12) {
     // ================= consumers: two groups of four warps, each serving BOTH passes ==========
     // Group 0 owns TMEM buffer 0 of either pipeline (the even tiles a CTA sees), group 1 buffer
-    // 1.  A group takes whichever of its tiles is ready, pass 2 first, so the exponential unit
-    // of every scheduler always has two warps to draw from while either pass has work.
+    // 1, so the exponential unit of every scheduler has two warps to draw from.
     //   pass 1: thread = (query head, window query) row, running (max, sum of exp2) per chunk
     //   pass 2: thread = key, window-mean attention per query head, pooling, score, entropy
+    // The order in which a group takes its tiles is static: the pass-1 tile comes first while
+    // its first key lies at most lag_keys beyond the first key of the group's next pass-2
+    // tile.  Because lag_keys covers a whole head, every pass-1 tile of a head precedes, in
+    // every CTA, every pass-2 tile of that head or a later one: the wait for a head's
+    // statistics always ends.  The lag also bounds the K bytes between the two passes (L2).
     constexpr int NH = 128 / W;  // query heads that fit the 128 columns
     const int grp = (warp - 4) >> 2, quad = warp & 3, row = quad * 32 + lane;
     const int t_in_win = row % W;
@@ -689,6 +669,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     const float inv_w = 1.0f / (float)W;
     const float sc2 = g.scale_log2;
     const bool avg = g.pool_kind == LAVA_POOL_AVG;
+    const int nblk = (rows_valid + 31) >> 5;  // 32-column blocks of window queries in use
     const uint32_t gbar = smem_u32(&m->gsync[grp]);
     uint32_t gphase = 0;
     bool alive = true;
@@ -700,8 +681,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     };
 
     // ---- cursors over the CTA's chunks of both passes ---------------------------------------
-    long long c1 = blockIdx.x, n1 = 0, j1 = 0;
-    int t1 = 0, last1 = 0;
+    int c1 = blockIdx.x, t1 = 0, last1 = 0;
+    long long n1 = 0, j1 = 0;
     bool has1 = c1 < total1;
     Chunk k1;
     float mx = -INFINITY, z = 0.f;
@@ -711,17 +692,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       last1 = row < rows_valid ? min(k1.s.n, k1.s.prefix + t_in_win + 1) : 0;
     };
     if (has1) open1();
-    long long c2 = blockIdx.x, n2 = 0, j2 = 0;
-    int t2 = 0;
+    int c2 = blockIdx.x, t2 = 0;
+    long long n2 = 0, j2 = 0;
     bool has2 = c2 < total2, prepped = false;
     Chunk k2;
     float es = 0.f, et = 0.f;  // entropy sums of this thread's keys over the chunk
     if (has2) k2 = decode_chunk(p, m, c2, 2);
-    if (grp == 0 && row == 0 && has2)
-      m->p2_pos = key_pos(p, k2.head, (long long)k2.tile0 * p.out_keys);
 
-    uint32_t idle = 0;
-    long long idle_t0 = 0;
     while (alive) {
       // ---- move the pass-1 cursor to this group's next tile; close finished chunks ----------
       while (has1 && alive) {
@@ -751,36 +728,18 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       // ---- the same for pass 2 ----------------------------------------------------------------
       while (has2 && alive) {
         if (t2 == k2.ntiles) {
-          // entropy sums of the chunk in a fixed order: keys of a thread, lanes, then warps
+          // entropy sums of the chunk in a fixed order: keys of a thread, lanes of a warp; the
+          // eight warp sums of a chunk are added up, in order, by the finishing kernel
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
             es += __shfl_down_sync(0xffffffffu, es, o);
             et += __shfl_down_sync(0xffffffffu, et, o);
           }
           if (lane == 0) {
-            m->red[grp][0][quad] = es;
-            m->red[grp][1][quad] = et;
-          }
-          group_sync();
-          if (!alive) break;
-          if (row == 0) {
-            const float(*r)[4] = m->red[grp];
-            const double s_sum = ((double)r[0][0] + (double)r[0][1]) + ((double)r[0][2] + (double)r[0][3]);
-            const double t_sum = ((double)r[1][0] + (double)r[1][1]) + ((double)r[1][2] + (double)r[1][3]);
-            p.ent_part[((size_t)k2.head * p.cph2_max + k2.index) * 2 + grp] = make_double2(s_sum, t_sum);
+            p.ent_part[((size_t)k2.head * p.cph2_max + k2.index) * 8 + grp * 4 + quad] =
+                make_float2(es, et);
             mbar_arrive(smem_u32(&m->prep_empty[j2 & 1]));
-            if (grp == 0) {
-              // the throttle of pass 1 follows the first key this CTA has still to score
-              long long next = 0x3fffffffffffffffLL;
-              if (c2 + gridDim.x < total2) {
-                const Chunk nx = decode_chunk(p, m, c2 + gridDim.x, 2);
-                next = key_pos(p, nx.head, (long long)nx.tile0 * p.out_keys);
-              }
-              m->p2_pos = next;
-            }
           }
-          group_sync();  // red[] is free again
-          if (!alive) break;
           es = 0.f;
           et = 0.f;
           prepped = false;
@@ -797,135 +756,16 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       }
       if (!alive || (!has1 && !has2)) break;
 
-      bool did = false;
-      // ---- a pass-2 tile: scores of 128 - 2 * pool_radius keys ----------------------------------
-      if (has2) {
-        if (!prepped)
-          prepped = __all_sync(0xffffffffu, mbar_test(smem_u32(&m->prep_full[j2 & 1]),
-                                                      (uint32_t)((j2 >> 1) & 1)));
-        if (prepped && __all_sync(0xffffffffu, mbar_test(smem_u32(&m->s2_full[grp]),
-                                                         (uint32_t)((n2 >> 1) & 1)))) {
-          did = true;
-          const Prep* prep = &m->prep[j2 & 1];
-          const int tile = k2.tile0 + t2;
-          tc_fence_after();
-          float acc[NH];
-#pragma unroll
-          for (int h = 0; h < NH; ++h) acc[h] = 0.f;
-          const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)grp * 128u;
-          // window queries come in blocks of 32 columns; a block lies inside one query head
-          // when W >= 32, and holds two heads when W == 16
-          const int nblk = (rows_valid + 31) >> 5;
-#pragma unroll 1
-          for (int blk = 0; blk < nblk; ++blk) {
-            float cur[32], l[32];
-            tmem_ld32_issue(taddr + blk * 32, cur);
-            // the block's log-sum-exp values travel to registers while the TMEM load is in flight
-#pragma unroll
-            for (int c4 = 0; c4 < 32; c4 += 4) {
-              const float4 l4 = *reinterpret_cast<const float4*>(&prep->lse[blk * 32 + c4]);
-              l[c4 + 0] = l4.x;
-              l[c4 + 1] = l4.y;
-              l[c4 + 2] = l4.z;
-              l[c4 + 3] = l4.w;
-            }
-            tmem_ld_wait(cur);
-            // stage by stage, so that independent operations follow one another in issue order
-#pragma unroll
-            for (int i = 0; i < 32; ++i) cur[i] = fmaf(cur[i], sc2, l[i]);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i]);
-            if (W >= 32) {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) cur[i] += cur[i + 16];
-#pragma unroll
-              for (int i = 0; i < 8; ++i) cur[i] += cur[i + 8];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) cur[i] += cur[i + 4];
-              const float sum = (cur[0] + cur[1]) + (cur[2] + cur[3]);
-              const int h = (blk * 32) / W;
-#pragma unroll
-              for (int hh = 0; hh < NH; ++hh)
-                if (hh == h) acc[hh] += sum;
-            } else {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                cur[i] += cur[i + 8];
-                cur[16 + i] += cur[24 + i];
-              }
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                cur[i] += cur[i + 4];
-                cur[16 + i] += cur[20 + i];
-              }
-              const float s0 = (cur[0] + cur[1]) + (cur[2] + cur[3]);
-              const float s1 = (cur[16] + cur[17]) + (cur[18] + cur[19]);
-#pragma unroll
-              for (int hh = 0; hh < NH; hh += 2)
-                if (hh == 2 * blk) {
-                  acc[hh] += s0;
-                  if (hh + 1 < NH) acc[hh + 1] += s1;
-                }
-            }
-          }
-          tc_fence_before();
-          mbar_arrive(smem_u32(&m->s2_empty[grp]));
-          // lane <-> key: the tile starts pool_radius keys before the first key it owns; keys
-          // outside the prefix hold the neutral element of both pools (values are >= 0)
-          const int ab = (int)((n2 >> 1) & 1);
-          const int key0 = tile * p.out_keys - rad;
-          const int i = key0 + row;
-          const bool inside = i >= 0 && i < k2.s.prefix;
-          float(*abuf)[kTile] = m->a[grp][ab];
-          if (avg) {
-#pragma unroll
-            for (int h = 0; h < NH; ++h) abuf[h][row] = inside ? acc[h] * inv_w : 0.f;
-          } else {
-            // max-pooling commutes with the group maximum: reduce over the query heads first
-            float top = 0.f;
-#pragma unroll
-            for (int h = 0; h < NH; ++h)
-              if (h < g.group) top = fmaxf(top, acc[h] * inv_w);
-            abuf[0][row] = inside ? top : 0.f;
-          }
-          group_sync();
-          if (!alive) break;
-          const int own_lo = tile * p.out_keys, own_hi = min(k2.s.prefix, own_lo + p.out_keys);
-          if (i >= own_lo && i < own_hi) {
-            float best = 0.f;
-            if (avg) {
-              for (int h = 0; h < g.group; ++h) {
-                const float* a = &abuf[h][row];
-                float pv = 0.f;
-                for (int q = -rad; q <= rad; ++q) pv += a[q];
-                best = fmaxf(best, pv / (float)g.pool_kernel);
-              }
-            } else {
-              const float* a = &abuf[0][row];
-              if (rad == 3) {
-                best = fmaxf(fmaxf(fmaxf(a[-3], a[-2]), fmaxf(a[-1], a[0])),
-                             fmaxf(fmaxf(a[1], a[2]), a[3]));
-              } else {
-                best = a[0];
-                for (int q = 1; q <= rad; ++q) best = fmaxf(best, fmaxf(a[-q], a[q]));
-              }
-            }
-            const float sc = best * prep->scale;
-            p.scores[(size_t)k2.layer * g.total_scores + k2.s.score_off +
-                     (long long)k2.kvh * k2.s.prefix + i] = sc;
-            if (sc > 0.f) {
-              es += sc;
-              et += sc * __logf(sc);
-            }
-          }
-          ++t2;
-          ++n2;
-        }
-      }
-      // ---- a pass-1 tile: running softmax statistics of 128 keys --------------------------------
-      if (!did && has1 &&
-          __all_sync(0xffffffffu, mbar_test(smem_u32(&m->s1_full[grp]), (uint32_t)((n1 >> 1) & 1)))) {
-        did = true;
+      bool take1 = has1;
+      if (has1 && has2)
+        take1 = key_pos(p, k1.head, (long long)(k1.tile0 + t1) * kTile) <=
+                key_pos(p, k2.head, (long long)(k2.tile0 + t2) * p.out_keys) + p.lag_keys;
+
+      if (take1) {
+        // ---- a pass-1 tile: running softmax statistics of 128 keys ------------------------------
+        if (!__all_sync(0xffffffffu, wait_bar(smem_u32(&m->s1_full[grp]),
+                                              (uint32_t)((n1 >> 1) & 1), m, p.status)))
+          break;
         tc_fence_after();
         const int limit = max(0, min(kTile, last1 - (k1.tile0 + t1) * kTile));
         const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)grp * 128u;
@@ -982,21 +822,131 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         mbar_arrive(smem_u32(&m->s1_empty[grp]));
         ++t1;
         ++n1;
-      }
-      if (did) {
-        idle = 0;
       } else {
-        // nothing ready for this group: step aside for a moment (bounded)
-        if (idle++ == 0) idle_t0 = clock64();
-        if (m->abort_flag) break;
-        __nanosleep(kBackoffNs);
-        if (clock64() - idle_t0 > kWaitCycles) {
-          give_up(m, p.status);
-          break;
+        // ---- a pass-2 tile: scores of 128 - 2 * pool_radius keys --------------------------------
+        if (!prepped) {
+          if (!__all_sync(0xffffffffu, wait_bar(smem_u32(&m->prep_full[j2 & 1]),
+                                                (uint32_t)((j2 >> 1) & 1), m, p.status)))
+            break;
+          prepped = true;
         }
+        if (!__all_sync(0xffffffffu, wait_bar(smem_u32(&m->s2_full[grp]),
+                                              (uint32_t)((n2 >> 1) & 1), m, p.status)))
+          break;
+        const Prep* prep = &m->prep[j2 & 1];
+        const int tile = k2.tile0 + t2;
+        tc_fence_after();
+        float acc[NH];
+#pragma unroll
+        for (int h = 0; h < NH; ++h) acc[h] = 0.f;
+        const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)grp * 128u;
+        // window queries come in blocks of 32 columns; a block lies inside one query head when
+        // W >= 32, and holds two heads when W == 16
+#pragma unroll 1
+        for (int blk = 0; blk < nblk; ++blk) {
+          float cur[32], l[32];
+          tmem_ld32_issue(taddr + blk * 32, cur);
+          // the block's log-sum-exp values travel to registers while the TMEM load is in flight
+#pragma unroll
+          for (int c4 = 0; c4 < 32; c4 += 4) {
+            const float4 l4 = *reinterpret_cast<const float4*>(&prep->lse[blk * 32 + c4]);
+            l[c4 + 0] = l4.x;
+            l[c4 + 1] = l4.y;
+            l[c4 + 2] = l4.z;
+            l[c4 + 3] = l4.w;
+          }
+          tmem_ld_wait(cur);
+          // stage by stage, so that independent operations follow one another in issue order
+#pragma unroll
+          for (int i = 0; i < 32; ++i) cur[i] = fmaf(cur[i], sc2, l[i]);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i]);
+          if (W >= 32) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) cur[i] += cur[i + 16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cur[i] += cur[i + 8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cur[i] += cur[i + 4];
+            const float sum = (cur[0] + cur[1]) + (cur[2] + cur[3]);
+            const int h = (blk * 32) / W;
+#pragma unroll
+            for (int hh = 0; hh < NH; ++hh)
+              if (hh == h) acc[hh] += sum;
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              cur[i] += cur[i + 8];
+              cur[16 + i] += cur[24 + i];
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              cur[i] += cur[i + 4];
+              cur[16 + i] += cur[20 + i];
+            }
+            const float s0 = (cur[0] + cur[1]) + (cur[2] + cur[3]);
+            const float s1 = (cur[16] + cur[17]) + (cur[18] + cur[19]);
+#pragma unroll
+            for (int hh = 0; hh < NH; hh += 2)
+              if (hh == 2 * blk) {
+                acc[hh] += s0;
+                if (hh + 1 < NH) acc[hh + 1] += s1;
+              }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(smem_u32(&m->s2_empty[grp]));
+        // lane <-> key: the tile starts pool_radius keys before the first key it owns; keys
+        // outside the prefix hold the neutral element of both pools (values are >= 0)
+        const int ab = (int)((n2 >> 1) & 1);
+        const int i = tile * p.out_keys - rad + row;
+        const bool inside = i >= 0 && i < k2.s.prefix;
+        float(*abuf)[kTile] = m->a[grp][ab];
+        if (avg) {
+#pragma unroll
+          for (int h = 0; h < NH; ++h) abuf[h][row] = inside ? acc[h] * inv_w : 0.f;
+        } else {
+          // max-pooling commutes with the group maximum: reduce over the query heads first
+          float top = 0.f;
+#pragma unroll
+          for (int h = 0; h < NH; ++h)
+            if (h < g.group) top = fmaxf(top, acc[h] * inv_w);
+          abuf[0][row] = inside ? top : 0.f;
+        }
+        group_sync();
+        if (!alive) break;
+        const int own_lo = tile * p.out_keys, own_hi = min(k2.s.prefix, own_lo + p.out_keys);
+        if (i >= own_lo && i < own_hi) {
+          float best = 0.f;
+          if (avg) {
+            for (int h = 0; h < g.group; ++h) {
+              const float* a = &abuf[h][row];
+              float pv = 0.f;
+              for (int q = -rad; q <= rad; ++q) pv += a[q];
+              best = fmaxf(best, pv / (float)g.pool_kernel);
+            }
+          } else {
+            const float* a = &abuf[0][row];
+            if (rad == 3) {
+              best = fmaxf(fmaxf(fmaxf(a[-3], a[-2]), fmaxf(a[-1], a[0])),
+                           fmaxf(fmaxf(a[1], a[2]), a[3]));
+            } else {
+              best = a[0];
+              for (int q = 1; q <= rad; ++q) best = fmaxf(best, fmaxf(a[-q], a[q]));
+            }
+          }
+          const float sc = best * prep->scale;
+          p.scores[(size_t)k2.layer * g.total_scores + k2.s.score_off +
+                   (long long)k2.kvh * k2.s.prefix + i] = sc;
+          if (sc > 0.f) {
+            es += sc;
+            et += sc * __logf(sc);
+          }
+        }
+        ++t2;
+        ++n2;
       }
     }
-    if (grp == 0 && row == 0) m->p2_pos = 0x3fffffffffffffffLL;  // pass 1 is no longer held back
   } else if (warp >= 12 && warp < 12 + kVWarps) {
     // ================= value-norm warps: the V rows of the CTA's pass-1 chunks ===============
     // 224 threads, 16 per row.  Rows are taken in groups of 112 (8 loads of 16 B per thread);
@@ -1100,7 +1050,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
 
 // entropy of one (layer, sequence) from the per-chunk sums, folded in a fixed order
 __global__ void __launch_bounds__(256)
-entropy_finalize_sm100_kernel(Geom g, const double2* ent_part, int cph2_max, int chunk_keys,
+entropy_finalize_sm100_kernel(Geom g, const float2* ent_part, int cph2_max, int chunk_keys,
                               double* entropy, const float* vbar_in, const unsigned* vbar_bits,
                               float* vbar_out) {
   __shared__ double rs[8], rt[8];
@@ -1115,9 +1065,15 @@ entropy_finalize_sm100_kernel(Geom g, const double2* ent_part, int cph2_max, int
   double sum_s = 0.0, sum_t = 0.0;
   for (int i = threadIdx.x; i < total; i += 256) {
     const int kvh = i / used, t = i - kvh * used;
-    const double2* e = ent_part + (((size_t)prob * g.n_kv_heads + kvh) * cph2_max + t) * 2;
-    sum_s += e[0].x + e[1].x;  // the two consumer groups of the chunk
-    sum_t += e[0].y + e[1].y;
+    const float2* e = ent_part + (((size_t)prob * g.n_kv_heads + kvh) * cph2_max + t) * 8;
+    double cs = 0.0, ct = 0.0;  // the eight consumer warps of the chunk, in order
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      cs += (double)e[u].x;
+      ct += (double)e[u].y;
+    }
+    sum_s += cs;
+    sum_t += ct;
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -1215,7 +1171,7 @@ Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   l.off_lse = off;
   off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total);
   l.off_ent = off;
-  off = up256(off + sizeof(double2) * 2 * (size_t)l.heads_total * l.tiles2);
+  off = up256(off + sizeof(float2) * 8 * (size_t)l.heads_total * l.tiles2);
   l.total = off;
   return l;
 }
@@ -1269,8 +1225,9 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.out_keys = lay.out_keys;
   p.cph1_max = lay.tiles1;
   p.cph2_max = lay.tiles2;
-  // Pass 1 must be allowed to finish the head pass 2 is waiting for (one head = max_seqlen
-  // keys); two further rounds of chunks cover the time the head's statistics take to fold.
+  // A pass-1 tile precedes a pass-2 tile while it starts at most lag_keys beyond it.  One
+  // head (max_seqlen keys) makes every wait for a head's statistics end; a few further rounds
+  // of chunks cover the time those statistics take to be published and folded.
   p.lag_keys = (long long)g.max_seqlen + (long long)lag_rounds_setting() * sms * p.chunk_tiles * kTile;
   p.vbar_in = vbar_in;
   p.scores = scores;
@@ -1283,7 +1240,7 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.vbar_bits = reinterpret_cast<unsigned*>(p.vcount + lay.heads_total);
   p.part = reinterpret_cast<float*>(ws + lay.off_part);
   p.neg_lse = reinterpret_cast<float*>(ws + lay.off_lse);
-  p.ent_part = reinterpret_cast<double2*>(ws + lay.off_ent);
+  p.ent_part = reinterpret_cast<float2*>(ws + lay.off_ent);
   p.status = reinterpret_cast<unsigned*>(ws_base);  // the status word opens the workspace
 
   rc = check_cuda(cudaMemsetAsync(ws + lay.off_sync, 0, lay.sync_bytes, stream),
@@ -1302,6 +1259,8 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   if (rc != LAVA_OK) return rc;
   // an upper bound on the pass-1 chunks; CTAs beyond the real count find no work and exit
   const long long chunks = (long long)lay.heads_total * lay.tiles1;
+  if ((long long)lay.heads_total * (lay.tiles2 > lay.tiles1 ? lay.tiles2 : lay.tiles1) > 0x3fffffffLL)
+    return fail(LAVA_ERR_UNSUPPORTED, "too many chunks for the 32-bit chunk index");
   const int grid = (int)(chunks < sms ? chunks : sms);
   // Cooperative launch: the CTAs wait on one another's flags, so all must be resident at once.
   void* args[3] = {&map_q, &map_k, &p};
