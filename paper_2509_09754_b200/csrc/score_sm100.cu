@@ -1120,13 +1120,13 @@ EncodeTiledFn encode_fn() {
 
 size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
-// tiles per chunk: tuning knob (LAVA_SM100_CHUNK_TILES), default 4
+// tiles per chunk: tuning knob (LAVA_SM100_CHUNK_TILES), default 8
 int chunk_tiles_setting() {
   static int value = 0;
   if (!value) {
     const char* e = getenv("LAVA_SM100_CHUNK_TILES");
     const int v = e ? atoi(e) : 0;
-    value = (v >= 1 && v <= 64) ? v : 4;
+    value = (v >= 1 && v <= 64) ? v : 8;
   }
   return value;
 }
@@ -1160,18 +1160,18 @@ Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   const int r = chunk_tiles_setting();
   l.heads_total = n_layers * g.batch * g.n_kv_heads;
   l.out_keys = kTile - 2 * g.pool_radius;
-  l.tiles1 = ceil_div(ceil_div(g.max_seqlen, kTile), r);                       // chunks, pass 1
-  l.tiles2 = ceil_div(ceil_div(max(1, g.max_seqlen - g.window), l.out_keys), r);  // chunks, pass 2
+  l.chunks1 = ceil_div(ceil_div(g.max_seqlen, kTile), r);                       // chunks, pass 1
+  l.chunks2 = ceil_div(ceil_div(max(1, g.max_seqlen - g.window), l.out_keys), r);  // chunks, pass 2
   size_t off = 0;
   l.off_sync = off;   // counters, ready flags, value-norm counters and bits: zeroed every launch
   off = up256(off + sizeof(int) * 4 * (size_t)l.heads_total);
   l.sync_bytes = off;
   l.off_part = off;
-  off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total * l.tiles1);
+  off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total * l.chunks1);
   l.off_lse = off;
   off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total);
   l.off_ent = off;
-  off = up256(off + sizeof(float2) * 8 * (size_t)l.heads_total * l.tiles2);
+  off = up256(off + sizeof(float2) * 8 * (size_t)l.heads_total * l.chunks2);
   l.total = off;
   return l;
 }
@@ -1223,8 +1223,8 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.n_layers = n_layers;
   p.chunk_tiles = chunk_tiles_setting();
   p.out_keys = lay.out_keys;
-  p.cph1_max = lay.tiles1;
-  p.cph2_max = lay.tiles2;
+  p.cph1_max = lay.chunks1;
+  p.cph2_max = lay.chunks2;
   // A pass-1 tile precedes a pass-2 tile while it starts at most lag_keys beyond it.  One
   // head (max_seqlen keys) makes every wait for a head's statistics end; a few further rounds
   // of chunks cover the time those statistics take to be published and folded.
@@ -1258,8 +1258,8 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
                                        (int)kSmemBytes), "cudaFuncSetAttribute(sm100 score)");
   if (rc != LAVA_OK) return rc;
   // an upper bound on the pass-1 chunks; CTAs beyond the real count find no work and exit
-  const long long chunks = (long long)lay.heads_total * lay.tiles1;
-  if ((long long)lay.heads_total * (lay.tiles2 > lay.tiles1 ? lay.tiles2 : lay.tiles1) > 0x3fffffffLL)
+  const long long chunks = (long long)lay.heads_total * lay.chunks1;
+  if ((long long)lay.heads_total * (lay.chunks2 > lay.chunks1 ? lay.chunks2 : lay.chunks1) > 0x3fffffffLL)
     return fail(LAVA_ERR_UNSUPPORTED, "too many chunks for the 32-bit chunk index");
   const int grid = (int)(chunks < sms ? chunks : sms);
   // Cooperative launch: the CTAs wait on one another's flags, so all must be resident at once.
@@ -1268,7 +1268,7 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
                                               kSmemBytes, stream), "score (sm100) launch");
   if (rc != LAVA_OK) return rc;
   entropy_finalize_sm100_kernel<<<n_layers * g.batch, 256, 0, stream>>>(
-      g, p.ent_part, lay.tiles2, p.chunk_tiles * lay.out_keys, entropy, vbar_in, p.vbar_bits,
+      g, p.ent_part, lay.chunks2, p.chunk_tiles * lay.out_keys, entropy, vbar_in, p.vbar_bits,
       vbar_out);
   count_launches(2);
   return check_cuda(cudaGetLastError(), "entropy finalize launch");
