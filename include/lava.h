@@ -133,6 +133,34 @@ LAVA_API lava_status lava_score_layers(const lava_layer_desc* desc, int32_t n_la
                               double* entropy, void* workspace, size_t workspace_bytes,
                               void* stream);
 
+/* The score step of one layer for callers that cannot allocate device memory (no counterpart
+ * in the paper: it exists for the callers, not for the method).
+ *
+ * Who needs it: code that runs inside another framework's memory pool without access to its
+ * allocator, plugins whose host forbids device allocations after start-up, and serving loops
+ * that must not risk the stall an allocation can cause.  Such a caller has inputs and outputs
+ * but no spare buffer to pass as `workspace`.  Here the scratch is a fixed 8 MiB array inside
+ * the library image; every GPU that loads the library holds it until the process exits.
+ *
+ * Same computation, same arguments and same results as lava_score_layer, minus the workspace:
+ *   device_status_out  DEVICE uint32, may be NULL: receives the status word of this call
+ *                      (LAVA_DEV_* bits) once `stream` has run past the call
+ * Limits and rules:
+ *   - A layer whose lava_workspace_bytes(desc, 1) exceeds 8 MiB is rejected with
+ *     LAVA_ERR_WORKSPACE before anything is enqueued (about 128K tokens at 32/8 heads, d 128).
+ *   - The first call on a device looks up the array's device address (a host-side set-up step,
+ *     once per device, with that device current); make that first call before any stream
+ *     capture begins.
+ *   - All calls share the one array, and it keeps the contents of the previous call; the entry
+ *     point clears what must start at zero itself.  Two calls whose kernels overlap on the GPU
+ *     (different streams, or different host threads on the same device) race on it: keep calls
+ *     on one device ordered on one stream.
+ *   - It calls no allocator: no cudaMalloc/cudaFree, no allocating library routine. */
+LAVA_API lava_status lava_score_layer_static(const lava_layer_desc* desc, const void* q_win,
+                                    const void* k, const void* v, const float* vbar_in,
+                                    float* scores, float* vbar_out, double* entropy,
+                                    uint32_t* device_status_out, void* stream);
+
 /* Step 2 -- layer budgets (Algorithm 2: B_l = e_l / sum_l e_l * B), made integral.
  *   entropy          double [n_layers, batch]
  *   total_budget     int64 [batch]: model-wide budget of each sequence in KV-head rows,

@@ -63,6 +63,8 @@ def load_library():
     lib.lava_poll_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.lava_wo_norm.argtypes = [vp, i32, i64, i64, vp, vp]
     lib.lava_score_layer.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_score_layer_static.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.lava_score_layer_static.restype = i32
     lib.lava_score_layers.argtypes = [dp, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, sz, vp]
     lib.lava_layer_budgets.argtypes = [i32, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp]
     lib.lava_select_topk.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
@@ -193,6 +195,17 @@ def lava_score_layer(desc: LayerDesc, q_win, k, v, vbar_in, scores, vbar_out, en
         ctypes.byref(c), _ptr(q_win), _ptr(k), _ptr(v), _ptr(vbar_in), _ptr(scores),
         _ptr(vbar_out), _ptr(entropy), _ptr(workspace), workspace.numel() * workspace.element_size(),
         _stream(stream)))
+
+
+def lava_score_layer_static(desc: LayerDesc, q_win, k, v, vbar_in, scores, vbar_out, entropy,
+                            device_status_out=None, stream=None) -> None:
+    """lava_score_layer without a workspace argument, for callers that cannot allocate device
+    memory (the scratch is an 8 MiB array inside the library; larger layers are rejected).
+    Calls on one device must not overlap on the GPU: keep them on one stream."""
+    c = desc.to_c()
+    _check(load_library().lava_score_layer_static(
+        ctypes.byref(c), _ptr(q_win), _ptr(k), _ptr(v), _ptr(vbar_in), _ptr(scores),
+        _ptr(vbar_out), _ptr(entropy), _ptr(device_status_out), _stream(stream)))
 
 
 def lava_score_layers(desc: LayerDesc, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
