@@ -248,6 +248,19 @@ __device__ inline uint4 ld_stream16(const void* p, uint64_t policy) {
   return r;
 }
 
+// D (+)= A * B on the register-operand tensor path: A 16 x 16 bf16 (row-major fragment a0..a3),
+// B 16 x 8 bf16 (b0, b1), D 16 x 8 fp32.  Thread (g = lane / 4, t = lane % 4) holds d0, d1 of
+// row g and d2, d3 of row g + 8; a0, a2 belong to row g and a1, a3 to row g + 8.
+__device__ inline void mma_bf16_16816(float& d0, float& d1, float& d2, float& d3, uint32_t a0,
+                                      uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                      uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+      "{%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 B apart.
 __device__ inline uint64_t make_desc(uint32_t saddr) {
   uint64_t d = 0;
@@ -949,18 +962,23 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     }
   } else if (warp >= 12 && warp < 12 + kVWarps) {
     // ================= value-norm warps: the V rows of the CTA's pass-1 chunks ===============
-    // 224 threads, 16 per row.  Rows are taken in groups of 112 (8 loads of 16 B per thread);
-    // one group is in flight while the previous one is reduced, across chunk borders too.
+    // Row L1 norms through the register-operand tensor path: a warp takes 16 rows at a time,
+    // clears the sign bits of the packed bf16 values and multiplies the 16 x 128 slab by a matrix
+    // of ones (mma.sync m16n8k16, fp32 accumulate, exact products), which leaves the row sums in
+    // the accumulator.  Which of a row's values lands in which k slot does not matter for a
+    // sum, so every thread simply loads 16-byte pieces: thread (g, t) of a warp, g = lane / 4,
+    // t = lane % 4, owns pieces t, t+4, t+8, t+12 of rows g and g+8.  Seven warps cover 112 rows
+    // per step; one step is in flight while the previous one is reduced.
     if (!p.vbar_in) {
       const uint64_t drop = policy_evict_first();
-      const int vt = threadIdx.x - 12 * 32;       // 0..223
-      const int sub = vt >> 4, piece = vt & 15;
+      const int vw = warp - 12;                   // 0..6
+      const int gq = lane >> 2, tq = lane & 3;
       struct Group {
-        const char* base;  // this thread's 16 bytes of row 0 of the sequence
+        const char* base;  // this thread's first 16 bytes of row 0 of the sequence
         int row0, row_hi, head;
         bool last;         // last group of its chunk
       };
-      long long c = blockIdx.x;
+      int c = blockIdx.x;
       Chunk ck;
       int grp = 0, ngrp = 0;
       auto next_group = [&](Group& gr) -> bool {
@@ -972,48 +990,40 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           ngrp = ceil_div(min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile) - ck.tile0 * kTile, 8 * kVRows);
         }
         gr.base = p.v + ((size_t)ck.layer * p.v_ls + (long long)ck.kvh * g.v_sh +
-                         ck.s.tok0 * g.v_st) * 2 + piece * 16;
-        gr.row0 = ck.tile0 * kTile + grp * 8 * kVRows + sub;
+                         ck.s.tok0 * g.v_st) * 2 + tq * 16;
+        gr.row0 = ck.tile0 * kTile + grp * 8 * kVRows + vw * 16 + gq;
         gr.row_hi = min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile);
         gr.head = ck.head;
         gr.last = ++grp == ngrp;
         return true;
       };
+      // buf[0..3]: pieces of row g, buf[4..7]: pieces of row g + 8 (zeros beyond the chunk)
       auto issue = [&](uint4 (&buf)[8], const Group& gr) {
 #pragma unroll
-        for (int s8 = 0; s8 < 8; ++s8) {
-          const int row = gr.row0 + s8 * kVRows;
-          buf[s8] = make_uint4(0, 0, 0, 0);
-          if (row < gr.row_hi) buf[s8] = ld_stream16(gr.base + (long long)row * g.v_st * 2, drop);
+        for (int half = 0; half < 2; ++half) {
+          const int row = gr.row0 + half * 8;
+          const char* src = gr.base + (long long)row * g.v_st * 2;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            buf[half * 4 + q] = make_uint4(0, 0, 0, 0);
+            if (row < gr.row_hi) buf[half * 4 + q] = ld_stream16(src + q * 64, drop);
+          }
         }
       };
       float best = 0.f;
+      const uint32_t ones = 0x3f803f80u;  // bf16 (1, 1)
       auto reduce = [&](const uint4 (&buf)[8], const Group& gr) {
-        float ps[8];
+        float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;  // d0: row g, d2: row g + 8
 #pragma unroll
-        for (int s8 = 0; s8 < 8; ++s8) {
-          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&buf[s8]);
-          float sum = 0.f;
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float2 f = __bfloat1622float2(h2[q]);
-            sum += fabsf(f.x) + fabsf(f.y);
-          }
-          ps[s8] = sum;
+        for (int q = 0; q < 4; ++q) {
+          const uint4 lo = buf[q], hi = buf[4 + q];
+          // two k = 16 steps per pair of pieces: (x, y) and (z, w)
+          mma_bf16_16816(d0, d1, d2, d3, lo.x & 0x7fff7fffu, hi.x & 0x7fff7fffu,
+                         lo.y & 0x7fff7fffu, hi.y & 0x7fff7fffu, ones, ones);
+          mma_bf16_16816(d0, d1, d2, d3, lo.z & 0x7fff7fffu, hi.z & 0x7fff7fffu,
+                         lo.w & 0x7fff7fffu, hi.w & 0x7fff7fffu, ones, ones);
         }
-        // eight row sums over the 16 lanes of a row in 8 shuffles: every step halves the rows
-        // a lane still carries and doubles the lanes folded into them
-        const bool b3 = (lane & 8) != 0, b2 = (lane & 4) != 0, b1 = (lane & 2) != 0;
-        float k4[4], k2[2];
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          k4[q] = (b3 ? ps[q + 4] : ps[q]) + __shfl_xor_sync(0xffffffffu, b3 ? ps[q] : ps[q + 4], 8);
-#pragma unroll
-        for (int q = 0; q < 2; ++q)
-          k2[q] = (b2 ? k4[q + 2] : k4[q]) + __shfl_xor_sync(0xffffffffu, b2 ? k4[q] : k4[q + 2], 4);
-        float k1 = (b1 ? k2[1] : k2[0]) + __shfl_xor_sync(0xffffffffu, b1 ? k2[0] : k2[1], 2);
-        k1 += __shfl_xor_sync(0xffffffffu, k1, 1);
-        best = fmaxf(best, k1);
+        best = fmaxf(best, fmaxf(d0, d2));
         if (gr.last) {  // warp-uniform
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
