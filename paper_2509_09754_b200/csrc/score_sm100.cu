@@ -45,16 +45,23 @@ constexpr uint32_t kHalfBytes = kTileBytes / 2;
 constexpr long long kWaitCycles = 1ll << 32;  // every wait gives up after about two seconds
 
 // shared memory map (bytes from a 1024-aligned base)
-constexpr uint32_t kOffQ1 = 0;
+// Two small operands in the un-swizzled K-major layout (8 x 16-byte core matrices, 128 B apart
+// along the rows, 2048 B apart along k) feed one extra k-step of every pass-2 tile: a [128 x 16]
+// tile whose first three columns are ones, and per head a [128 x 16] tile that carries, per window
+// query, minus its log2-sum-exp (in logit units) split into three bf16 terms.  The MMA thereby
+// adds the softmax normaliser to every logit, and the score warps need no per-column constants.
+constexpr uint32_t kOffOnes = 0;
+constexpr uint32_t kOffBias = 4096;          // two slots of 4 KB
+constexpr uint32_t kSmallTileBytes = 4096;
+constexpr uint32_t kOffQ1 = 16384;
 constexpr uint32_t kOffQ2 = kOffQ1 + kTileBytes;
 constexpr uint32_t kOffK1 = kOffQ2 + kTileBytes;
 constexpr uint32_t kOffK2 = kOffK1 + kStages * kTileBytes;
-constexpr uint32_t kOffMisc = kOffK2 + kStages * kTileBytes;  // 192 KB
-constexpr uint32_t kMiscBytes = 26624;
+constexpr uint32_t kOffMisc = kOffK2 + kStages * kTileBytes;  // 16 KB + 192 KB
+constexpr uint32_t kMiscBytes = 15360;
 constexpr uint32_t kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + alignment slack
 
 struct Prep {                 // what the score warps need to know about a head
-  alignas(16) float lse[128]; // -(log2-sum-exp) per window query
   float scale;                // Vbar * c_hat
   float pad[3];
 };
@@ -71,7 +78,7 @@ struct Misc {
   int sched_total1, sched_total2;     // chunks per layer of pass 1 / pass 2
   alignas(16) float pub[2][2][128];   // [slot][group][query]: log2-sum-exp of a finished chunk
   Prep prep[2];
-  alignas(16) float a[2][2][8][kTile];  // [group][tile parity][query head][key]: window means
+  alignas(16) float a[2][2][4][kTile];  // [group][tile parity][query head][key]: window means
   int pref1[kMaxBatch + 1], pref2[kMaxBatch + 1];  // exclusive scans of chunks per sequence
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
@@ -271,6 +278,16 @@ __device__ inline uint64_t make_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;            // 128-byte swizzle
   return d;
 }
+// The same for an un-swizzled K-major operand of 16 columns: core matrices of 8 rows x 16 bytes,
+// 2048 B apart along k (leading offset) and 128 B apart along the rows (stride offset).
+__device__ inline uint64_t make_desc_plain(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(2048 >> 4) << 16;
+  d |= (uint64_t)(128 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
@@ -425,6 +442,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  // ones tile: columns 0..2 of every row hold bf16 1.0; bias tiles start as zeros
+  for (int i = threadIdx.x; i < (int)(3 * kSmallTileBytes / 16); i += kThreads) {
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (i < 128) val = make_uint4(0x3f803f80u, 0x00003f80u, 0, 0);  // k-core 0 of row i
+    *reinterpret_cast<uint4*>(gen + kOffOnes + i * 16) = val;
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 2) tmem_alloc(smem_u32(&m->tmem_base), 512);
   tc_fence_before();
   __syncthreads();
@@ -497,9 +521,25 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
+      // per window query: minus the log2-sum-exp in logit units, as three bf16 terms
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        m->prep[slot].lse[lane + 32 * q] = __ldcg(p.neg_lse + (size_t)ck.head * 128 + lane + 32 * q);
+      for (int q = 0; q < 4; ++q) {
+        const int r = lane + 32 * q;
+        const float nl = __ldcg(p.neg_lse + (size_t)ck.head * 128 + r);
+        uint32_t w0 = 0xf149u, w1 = 0;  // about -1e30 for a query without any key
+        if (nl > -INFINITY) {
+          const float b = nl / g.scale_log2;
+          const __nv_bfloat16 b0 = __float2bfloat16_rn(b);
+          const float r1 = b - __bfloat162float(b0);
+          const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
+          const __nv_bfloat16 b2 = __float2bfloat16_rn(r1 - __bfloat162float(b1));
+          w0 = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
+          w1 = (uint32_t)__bfloat16_as_ushort(b2);
+        }
+        *reinterpret_cast<uint4*>(gen + kOffBias + slot * kSmallTileBytes + (r >> 3) * 128 +
+                                  (r & 7) * 16) = make_uint4(w0, w1, 0, 0);
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       if (lane == 0) {
         const float vb = p.vbar_in ? p.vbar_in[ck.head]
                                    : __uint_as_float(__ldcg(p.vbar_bits + ck.head));
@@ -561,7 +601,10 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       bool ok = true;
       for (long long c = blockIdx.x; c < total && ok; c += gridDim.x) {
         const int nt = decode_chunk(p, m, c, pass).ntiles;
+        const int slot = q_uses & 1;  // chunk ordinal parity = slot of the head's bias tile
         ok = wait_bar(q_full, (uint32_t)(q_uses & 1), m, p.status);
+        if (ok && !first)
+          ok = wait_bar(smem_u32(&m->prep_full[slot]), (uint32_t)((q_uses >> 1) & 1), m, p.status);
         ++q_uses;
         for (int t = 0; t < nt && ok; ++t, ++n) {
           const int st = (int)(n % kStages), buf = (int)(n & 1);
@@ -578,6 +621,10 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
             if (first) umma_bf16(d, make_desc(q_addr + off), make_desc(kt + off), kIdesc, kk > 0);
             else umma_bf16(d, make_desc(kt + off), make_desc(q_addr + off), kIdesc, kk > 0);
           }
+          // pass 2: one more k-step adds minus the log2-sum-exp of every window query
+          if (!first)
+            umma_bf16(d, make_desc_plain(base + kOffOnes),
+                      make_desc_plain(base + kOffBias + slot * kSmallTileBytes), kIdesc, 1);
           umma_commit(smem_u32(&k_empty[st]));
           umma_commit(smem_u32(&s_full[buf]));
         }
@@ -857,23 +904,12 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         // W >= 32, and holds two heads when W == 16
 #pragma unroll 1
         for (int blk = 0; blk < nblk; ++blk) {
-          float cur[32], l[32];
+          float cur[32];
           tmem_ld32_issue(taddr + blk * 32, cur);
-          // the block's log-sum-exp values travel to registers while the TMEM load is in flight
-#pragma unroll
-          for (int c4 = 0; c4 < 32; c4 += 4) {
-            const float4 l4 = *reinterpret_cast<const float4*>(&prep->lse[blk * 32 + c4]);
-            l[c4 + 0] = l4.x;
-            l[c4 + 1] = l4.y;
-            l[c4 + 2] = l4.z;
-            l[c4 + 3] = l4.w;
-          }
           tmem_ld_wait(cur);
-          // stage by stage, so that independent operations follow one another in issue order
+          // the MMA has already subtracted the log-sum-exp: p = exp2(scale * logit)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) cur[i] = fmaf(cur[i], sc2, l[i]);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i]);
+          for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i] * sc2);
           if (W >= 32) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) cur[i] += cur[i + 16];
@@ -917,7 +953,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         float(*abuf)[kTile] = m->a[grp][ab];
         if (avg) {
 #pragma unroll
-          for (int h = 0; h < NH; ++h) abuf[h][row] = inside ? acc[h] * inv_w : 0.f;
+          for (int h = 0; h < NH; ++h)
+            if (h < 4 && h < g.group) abuf[h][row] = inside ? acc[h] * inv_w : 0.f;
         } else {
           // max-pooling commutes with the group maximum: reduce over the query heads first
           float top = 0.f;
@@ -1160,6 +1197,7 @@ bool sm100_supported(const Geom& g) {
   if (g.dtype != LAVA_BF16 || g.head_dim != 128) return false;
   if (g.window != 16 && g.window != 32 && g.window != 64 && g.window != 128) return false;
   if (g.group * g.window > 128 || g.group > 8) return false;
+  if (g.pool_kind == LAVA_POOL_AVG && g.group > 4) return false;  // room for 4 heads' window means
   if (g.pool_radius > 31) return false;
   if (g.batch > kMaxBatch) return false;
   return true;
