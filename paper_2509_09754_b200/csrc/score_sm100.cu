@@ -76,6 +76,7 @@ struct Misc {
   uint32_t tmem_base;
   volatile int abort_flag;
   int sched_total1, sched_total2;     // chunks per layer of pass 1 / pass 2
+  int lead_tiles;                     // tile slots pass 1 runs ahead of pass 2 in a CTA's order
   alignas(16) float pub[2][2][128];   // [slot][group][query]: log2-sum-exp of a finished chunk
   Prep prep[2];
   alignas(16) float a[2][2][4][kTile];  // [group][tile parity][query head][key]: window means
@@ -89,7 +90,7 @@ struct Sm100Params {
   int chunk_tiles;          // tiles per chunk
   int out_keys;             // keys a pass-2 tile owns: 128 - 2 * pool_radius
   int cph1_max, cph2_max;   // chunks per head at max_seqlen (strides of the scratch arrays)
-  long long lag_keys;       // a pass-1 tile may start this many keys beyond the next pass-2 tile
+  int lead_extra;           // tiles pass 1 leads pass 2 by, beyond what head completion needs
   const float* vbar_in;
   float* scores;
   float* vbar_out;
@@ -351,11 +352,6 @@ __device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, int c,
   return ck;
 }
 
-// global key coordinate that orders the tiles of the two passes
-__device__ inline long long key_pos(const Sm100Params& p, int head, long long key) {
-  return (long long)head * p.g.max_seqlen + key;
-}
-
 // ------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------
@@ -411,6 +407,20 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     if (threadIdx.x == 0) {
       m->sched_total1 = g.n_kv_heads * m->pref1[g.batch];
       m->sched_total2 = g.n_kv_heads * m->pref2[g.batch];
+      // How far pass 1 must lead pass 2 in a CTA's own order (see the consumer warps).  With
+      // rho = pass-2 chunks per pass-1 chunk: rho * (1 + (longest head + drift) / grid) chunks,
+      // where drift is how far the two passes' chunk numbering can diverge inside a layer.
+      const double t1 = (double)m->sched_total1, t2 = (double)m->sched_total2;
+      const double rho = t1 > 0.0 ? t2 / t1 : 1.0;
+      double drift = 0.0, longest = 0.0;
+      for (int b = 0; b < g.batch; ++b) {
+        const double c1 = m->pref1[b + 1] - m->pref1[b], c2 = m->pref2[b + 1] - m->pref2[b];
+        const double at = fabs(g.n_kv_heads * (m->pref1[b] * rho - m->pref2[b]));
+        drift = fmax(drift, at + g.n_kv_heads * fabs(c1 * rho - c2));
+        longest = fmax(longest, c1);
+      }
+      const double lead = p.chunk_tiles * rho * (1.0 + (longest + drift) / (double)gridDim.x);
+      m->lead_tiles = (int)ceil(lead) + p.lead_extra;
     }
   }
 
@@ -717,11 +727,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     // 1, so the exponential unit of every scheduler has two warps to draw from.
     //   pass 1: thread = (query head, window query) row, running (max, sum of exp2) per chunk
     //   pass 2: thread = key, window-mean attention per query head, pooling, score, entropy
-    // The order in which a group takes its tiles is static: the pass-1 tile comes first while
-    // its first key lies at most lag_keys beyond the first key of the group's next pass-2
-    // tile.  Because lag_keys covers a whole head, every pass-1 tile of a head precedes, in
-    // every CTA, every pass-2 tile of that head or a later one: the wait for a head's
-    // statistics always ends.  The lag also bounds the K bytes between the two passes (L2).
+    // The order in which the tiles are taken is static and alternates tile by tile: counting a
+    // CTA's tiles in slots (chunk ordinal * chunk_tiles + tile), the pass-1 tile comes first
+    // while its slot, scaled to pass-2 slots, is at most lead_tiles beyond the next pass-2
+    // slot.  The lead is long enough that every pass-1 chunk of a head precedes, in every CTA,
+    // every pass-2 tile of that head or a later one, so the wait for a head's statistics
+    // always ends; it is short enough to keep the K tiles between the two passes in L2, and the
+    // fine alternation keeps both TMA/MMA pipelines busy all the time.
     constexpr int NH = 128 / W;  // query heads that fit the 128 columns
     const int grp = (warp - 4) >> 2, quad = warp & 3, row = quad * 32 + lane;
     const int t_in_win = row % W;
@@ -818,8 +830,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
 
       bool take1 = has1;
       if (has1 && has2)
-        take1 = key_pos(p, k1.head, (long long)(k1.tile0 + t1) * kTile) <=
-                key_pos(p, k2.head, (long long)(k2.tile0 + t2) * p.out_keys) + p.lag_keys;
+        take1 = (j1 * p.chunk_tiles + t1) * (long long)m->sched_total2 <=
+                (j2 * p.chunk_tiles + t2 + m->lead_tiles) * (long long)m->sched_total1;
 
       if (take1) {
         // ---- a pass-1 tile: running softmax statistics of 128 keys ------------------------------
@@ -1179,14 +1191,14 @@ int chunk_tiles_setting() {
 }
 
 
-// rounds of chunks pass 1 may run ahead of a head's completion: tuning knob
-// (LAVA_SM100_LAG_ROUNDS), default 2
-int lag_rounds_setting() {
+// tiles pass 1 leads pass 2 by beyond what head completion needs (covers the time a head's
+// statistics take to be published and folded): tuning knob (LAVA_SM100_LEAD_TILES), default 3
+int lead_extra_setting() {
   static int value = -1;
   if (value < 0) {
-    const char* e = getenv("LAVA_SM100_LAG_ROUNDS");
+    const char* e = getenv("LAVA_SM100_LEAD_TILES");
     const int v = e ? atoi(e) : -1;
-    value = (v >= 0 && v <= 4096) ? v : 2;
+    value = (v >= 0 && v <= 4096) ? v : 3;
   }
   return value;
 }
@@ -1273,10 +1285,7 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.out_keys = lay.out_keys;
   p.cph1_max = lay.chunks1;
   p.cph2_max = lay.chunks2;
-  // A pass-1 tile precedes a pass-2 tile while it starts at most lag_keys beyond it.  One
-  // head (max_seqlen keys) makes every wait for a head's statistics end; a few further rounds
-  // of chunks cover the time those statistics take to be published and folded.
-  p.lag_keys = (long long)g.max_seqlen + (long long)lag_rounds_setting() * sms * p.chunk_tiles * kTile;
+  p.lead_extra = lead_extra_setting();
   p.vbar_in = vbar_in;
   p.scores = scores;
   p.vbar_out = vbar_out;
