@@ -8,8 +8,7 @@
 //       one thread per row reads its TMEM lane and keeps a running (max, sum of exp2) over the
 //       keys the query may see (Sec. 2: softmax over i <= j).  Work is dealt to CTAs in chunks
 //       of a few consecutive tiles of one head; a chunk's statistics leave the CTA once, through
-//       a publisher warp.  The publisher that completes a head folds the chunk partials, in
-//       chunk order, into one log-sum-exp per query and raises the head's ready flag.  Seven
+//       a publisher warp that also counts the head's published chunks.  Seven
 //       more warps stream the chunk's V rows for the value norm (Theorem 1: max_k ||V[k]||_1).
 //   pass 2 (scores)      S^T = K Q_g^T (rows = keys, columns = window queries)
 //       one thread per key: a_h[i] = (1/w) sum_t exp2(z - lse_t) per query head in registers,
@@ -23,7 +22,7 @@
 //
 // K is read from HBM once: pass 2 trails pass 1 by a bounded number of keys, so its tiles are
 // still in L2 (K tiles are loaded with an evict-last hint in pass 1 and evict-first in pass 2,
-// V rows with evict-first).  Every wait (mbarrier, ready flag, throttle) is bounded in time; on
+// V rows with evict-first).  Every wait (mbarrier, head counters) is bounded in time; on
 // expiry the kernel sets LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
 #include <cuda.h>
 #include <stdlib.h>
@@ -99,10 +98,8 @@ struct Sm100Params {
   // scratch
   float* part;              // [heads_total][cph1_max][128] log2-sum-exp per chunk and query
   int* counters;            // [heads_total] published pass-1 chunks
-  int* ready;               // [heads_total]
   int* vcount;              // [heads_total] finished value-norm warps
   unsigned* vbar_bits;      // [heads_total]
-  float* neg_lse;           // [heads_total][128]
   float2* ent_part;         // [heads_total][cph2_max][8 consumer warps] (sum s, sum s ln s)
   unsigned* status;
 };
@@ -234,11 +231,9 @@ __device__ inline float lse2(float a, float b) {
   return hi + fast_log2(1.0f + fast_exp2(lo - hi));
 }
 // counter increment that publishes this thread's earlier writes (and those ordered before it by
-// a barrier) and makes the writes of earlier incrementers visible to the caller
-__device__ inline int atom_add_acq_rel(int* p, int v) {
-  int old;
-  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
-  return old;
+// a barrier)
+__device__ inline void red_add_release(int* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ inline int ld_acquire(const int* p) {
   int v;
@@ -514,13 +509,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     for (long long c = blockIdx.x; c < total2; c += gridDim.x, ++j) {
       const Chunk ck = decode_chunk(p, m, c, 2);
       const int slot = (int)(j & 1);
-      // wait until the head's log-sum-exp and value norm are final
+      // wait until every pass-1 chunk of the head has been published and its value norm is final
       bool ok = true;
+      const int cph1 = ceil_div(ceil_div(ck.s.n, kTile), p.chunk_tiles);
       if (lane == 0) {
-        const int want_v =
-            p.vbar_in ? 0 : kVWarps * ceil_div(ceil_div(ck.s.n, kTile), p.chunk_tiles);
+        const int want_v = p.vbar_in ? 0 : kVWarps * cph1;
         const long long t0 = clock64();
-        while (ld_acquire(&p.ready[ck.head]) == 0 ||
+        while (ld_acquire(&p.counters[ck.head]) < cph1 ||
                (want_v && ld_acquire(&p.vcount[ck.head]) < want_v)) {
           if (m->abort_flag) break;
           __nanosleep(100);
@@ -531,23 +526,61 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
-      // per window query: minus the log2-sum-exp in logit units, as three bf16 terms
+      // Fold the head's chunk partials, in chunk order, into one log2-sum-exp per window query
+      // (lane l: queries 4l .. 4l+3).  Every CTA that scores a chunk of the head does this for
+      // itself, with the same operations in the same order, so all of them get the same bits
+      // and no CTA waits for another one's fold.
+      {
+        const float4* pp =
+            reinterpret_cast<const float4*>(p.part + (size_t)ck.head * p.cph1_max * 128) + lane;
+        float big[4], sum[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int r = lane + 32 * q;
-        const float nl = __ldcg(p.neg_lse + (size_t)ck.head * 128 + r);
-        uint32_t w0 = 0xf149u, w1 = 0;  // about -1e30 for a query without any key
-        if (nl > -INFINITY) {
-          const float b = nl / g.scale_log2;
-          const __nv_bfloat16 b0 = __float2bfloat16_rn(b);
-          const float r1 = b - __bfloat162float(b0);
-          const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
-          const __nv_bfloat16 b2 = __float2bfloat16_rn(r1 - __bfloat162float(b1));
-          w0 = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
-          w1 = (uint32_t)__bfloat16_as_ushort(b2);
+        for (int q = 0; q < 4; ++q) {
+          big[q] = -INFINITY;
+          sum[q] = 0.f;
         }
-        *reinterpret_cast<uint4*>(gen + kOffBias + slot * kSmallTileBytes + (r >> 3) * 128 +
-                                  (r & 7) * 16) = make_uint4(w0, w1, 0, 0);
+#pragma unroll 1
+        for (int i0 = 0; i0 < cph1; i0 += 16) {
+          float4 pr[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u)
+            pr[u] = (i0 + u < cph1) ? __ldcg(pp + (size_t)(i0 + u) * 32)
+                                    : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            float l[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u)
+              l[u] = q == 0 ? pr[u].x : q == 1 ? pr[u].y : q == 2 ? pr[u].z : pr[u].w;
+            float bm = l[0];
+#pragma unroll
+            for (int u = 1; u < 16; ++u) bm = fmaxf(bm, l[u]);
+            const float nb = fmaxf(big[q], bm);
+            const float ref = nb == -INFINITY ? 0.f : nb;  // keeps -inf - -inf out of the exponent
+            float acc = sum[q] * fast_exp2(big[q] - ref);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) acc += fast_exp2(l[u] - ref);
+            sum[q] = acc;
+            big[q] = nb;
+          }
+        }
+        // per window query: minus the log2-sum-exp in logit units, as three bf16 terms
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int r = 4 * lane + q;
+          uint32_t w0 = 0xf149u, w1 = 0;  // about -1e30 for a query without any key
+          if (sum[q] > 0.f) {
+            const float b = -(big[q] + fast_log2(sum[q])) / g.scale_log2;
+            const __nv_bfloat16 b0 = __float2bfloat16_rn(b);
+            const float r1 = b - __bfloat162float(b0);
+            const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 b2 = __float2bfloat16_rn(r1 - __bfloat162float(b1));
+            w0 = (uint32_t)__bfloat16_as_ushort(b0) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
+            w1 = (uint32_t)__bfloat16_as_ushort(b2);
+          }
+          *reinterpret_cast<uint4*>(gen + kOffBias + slot * kSmallTileBytes + r * 16) =
+              make_uint4(w0, w1, 0, 0);
+        }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       if (lane == 0) {
@@ -647,7 +680,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       wait_bar(smem_u32(drain), 0, m, p.status, false);
     }
   } else if (warp == 3) {
-    // ================= publisher: chunk statistics leave the CTA; head folding ===============
+    // ================= publisher: chunk statistics leave the CTA ============================
     long long j = 0;
     for (long long c = blockIdx.x; c < total1; c += gridDim.x, ++j) {
       const Chunk ck = decode_chunk(p, m, c, 1);
@@ -670,55 +703,10 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         reinterpret_cast<float4*>(dst)[lane] = o4;
       }
       __syncwarp();
-      int last = 0;
       if (lane == 0) {
         mbar_arrive(smem_u32(&m->pub_empty[slot]));
-        last = atom_add_acq_rel(&p.counters[ck.head], 1) == ck.cph - 1;
-      }
-      last = __shfl_sync(0xffffffffu, last, 0);
-      if (last) {
-        // fold the head's chunk partials, in chunk order, into one log-sum-exp per window query
-        const float4* pp =
-            reinterpret_cast<const float4*>(p.part + (size_t)ck.head * p.cph1_max * 128) + lane;
-        float big[4], sum[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          big[q] = -INFINITY;
-          sum[q] = 0.f;
-        }
-#pragma unroll 1
-        for (int i0 = 0; i0 < ck.cph; i0 += 16) {
-          float4 pr[16];
-#pragma unroll
-          for (int u = 0; u < 16; ++u)
-            pr[u] = (i0 + u < ck.cph) ? __ldcg(pp + (size_t)(i0 + u) * 32)
-                                      : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            float l[16];
-#pragma unroll
-            for (int u = 0; u < 16; ++u)
-              l[u] = q == 0 ? pr[u].x : q == 1 ? pr[u].y : q == 2 ? pr[u].z : pr[u].w;
-            float bm = l[0];
-#pragma unroll
-            for (int u = 1; u < 16; ++u) bm = fmaxf(bm, l[u]);
-            const float nb = fmaxf(big[q], bm);
-            const float ref = nb == -INFINITY ? 0.f : nb;  // keeps -inf - -inf out of the exponent
-            float acc = sum[q] * fast_exp2(big[q] - ref);
-#pragma unroll
-            for (int u = 0; u < 16; ++u) acc += fast_exp2(l[u] - ref);
-            sum[q] = acc;
-            big[q] = nb;
-          }
-        }
-        float4 out;
-        out.x = sum[0] > 0.f ? -(big[0] + fast_log2(sum[0])) : -INFINITY;
-        out.y = sum[1] > 0.f ? -(big[1] + fast_log2(sum[1])) : -INFINITY;
-        out.z = sum[2] > 0.f ? -(big[2] + fast_log2(sum[2])) : -INFINITY;
-        out.w = sum[3] > 0.f ? -(big[3] + fast_log2(sum[3])) : -INFINITY;
-        reinterpret_cast<float4*>(p.neg_lse + (size_t)ck.head * 128)[lane] = out;
-        __syncwarp();
-        if (lane == 0) st_release(&p.ready[ck.head], 1);
+        // release: the partial written above is visible to whoever sees the new count
+        red_add_release(&p.counters[ck.head], 1);
       }
     }
   } else if (warp >= 4 && warp < 12) {
@@ -1223,13 +1211,11 @@ Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   l.chunks1 = ceil_div(ceil_div(g.max_seqlen, kTile), r);                       // chunks, pass 1
   l.chunks2 = ceil_div(ceil_div(max(1, g.max_seqlen - g.window), l.out_keys), r);  // chunks, pass 2
   size_t off = 0;
-  l.off_sync = off;   // counters, ready flags, value-norm counters and bits: zeroed every launch
-  off = up256(off + sizeof(int) * 4 * (size_t)l.heads_total);
+  l.off_sync = off;   // chunk counters, value-norm counters and bits: zeroed every launch
+  off = up256(off + sizeof(int) * 3 * (size_t)l.heads_total);
   l.sync_bytes = off;
   l.off_part = off;
   off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total * l.chunks1);
-  l.off_lse = off;
-  off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total);
   l.off_ent = off;
   off = up256(off + sizeof(float2) * 8 * (size_t)l.heads_total * l.chunks2);
   l.total = off;
@@ -1292,11 +1278,9 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.v = (const char*)v;
   p.v_ls = v_ls;
   p.counters = reinterpret_cast<int*>(ws + lay.off_sync);
-  p.ready = p.counters + lay.heads_total;
-  p.vcount = p.ready + lay.heads_total;
+  p.vcount = p.counters + lay.heads_total;
   p.vbar_bits = reinterpret_cast<unsigned*>(p.vcount + lay.heads_total);
   p.part = reinterpret_cast<float*>(ws + lay.off_part);
-  p.neg_lse = reinterpret_cast<float*>(ws + lay.off_lse);
   p.ent_part = reinterpret_cast<float2*>(ws + lay.off_ent);
   p.status = reinterpret_cast<unsigned*>(ws_base);  // the status word opens the workspace
 
