@@ -95,12 +95,16 @@ select_topk_kernel(Geom g, const float* scores, const long long* layer_budget, i
         const unsigned key = i < c1 ? keys[i] : 0u;
         const bool mine = i < c1 && (key & prefix_mask) == prefix_val;
         const unsigned digit = (key >> shift) & dmask;
-        // one shared-memory atomic per distinct digit in the warp
+        // Scores of one layer crowd into a few exponent buckets, so most lanes of a row share
+        // the digit of the first active lane: those are counted by one atomic, the rest add
+        // their own (spread digits rarely collide).
         const unsigned active = __ballot_sync(0xffffffffu, mine);
-        if (mine) {
-          const unsigned peers = __match_any_sync(active, digit);
-          if ((threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1))
-            atomicAdd(&sh.hist[digit], (unsigned)__popc(peers));
+        if (active) {
+          const int leader = __ffs(active) - 1;
+          const unsigned d0 = __shfl_sync(0xffffffffu, digit, leader);
+          const unsigned same = __ballot_sync(0xffffffffu, mine && digit == d0);
+          if ((int)(threadIdx.x & 31) == leader) atomicAdd(&sh.hist[d0], (unsigned)__popc(same));
+          else if (mine && digit != d0) atomicAdd(&sh.hist[digit], 1u);
         }
       }
       cluster.sync();  // every CTA's histogram is complete
@@ -194,31 +198,45 @@ select_topk_kernel(Geom g, const float* scores, const long long* layer_budget, i
 
 
 // ------------------------------------------------------------------------------------------
-// Register-resident variant: every thread loads its E keys once and keeps them for all passes.
-// A warp owns E consecutive rows of 32 keys (row i, lane l <-> key base + 32 i + l), so loads
-// are coalesced and the element order inside a warp is (row, lane): exclusive counts along a
-// row come from one ballot, and no block-wide scan runs per 512 keys.  Serves problems of up to
-// 32768 keys per CTA (cluster of 8 or 16 CTAs); larger ones take the streaming kernel above.
+// Register-resident variant: every thread keeps E consecutive keys in registers for all passes,
+// so element order is thread order and nothing in the passes or the emit needs a warp vote.
+// Keys reach the registers through a padded shared-memory staging area (coalesced global reads,
+// conflict-free 16-byte shared reads).  The digit histogram is kept in kRep interleaved copies
+// (copy = lane mod kRep): layer scores crowd into a few exponent buckets, and a single copy
+// would serialise the shared-memory atomics of a warp on those few addresses.  Kept positions
+// are packed in shared memory and leave with coalesced stores.  Serves problems of up to 32768
+// keys per CTA (cluster of 8 or 16 CTAs); larger ones take the streaming kernel above.
 // ------------------------------------------------------------------------------------------
 constexpr int kRegMaxPerCta = 32768;
 
 struct RegShared {
-  unsigned hist[kBins];
-  unsigned total[kBins];
+  unsigned hist[kBins];    // this CTA's folded histogram; peers read it through DSMEM
+  unsigned total[kBins];   // cluster-wide histogram (peers write their share of the bins)
   unsigned warp_sum[kWarps + 1];
   unsigned found_digit, found_before;
-  uint2 warp_cnt[kWarps];   // (above tau, equal to tau) per warp of this CTA; peers read it
+  uint2 cta_cnt;           // (above tau, equal to tau) inside this CTA; peers read it
+};
+
+template <int E>
+struct RegCfg {
+  static constexpr int kRep = E >= 32 ? 16 : 4;  // histogram copies
+  static constexpr int kPad = E + 4;             // staging words per thread (bank spread)
+  static constexpr int kStageWords = kThreads * kPad;
+  static constexpr int kHistWords = kBins * kRep;
+  static constexpr int kBigWords = kStageWords > kHistWords ? kStageWords : kHistWords;
 };
 
 template <int E>
 __global__ void __launch_bounds__(kThreads)
 select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budget, int* keep_idx,
                        int* head_offsets) {
+  using Cfg = RegCfg<E>;
+  extern __shared__ __align__(16) unsigned big[];  // staging / histogram copies / packed output
   __shared__ RegShared sh;
   cg::cluster_group cluster = cg::this_cluster();
   const int csize = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const int prob = blockIdx.x / csize, layer = prob / g.batch, b = prob - layer * g.batch;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
   const SeqInfo s = seq_info(g, b);
   const int m_total = g.n_kv_heads * s.prefix;  // candidates (fits 31 bits)
   const unsigned* keys =
@@ -231,16 +249,28 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
   if (k_sel < 0) k_sel = 0;
   if (k_sel > m_total) k_sel = m_total;
 
-  // this CTA's range, and inside it this warp's E rows of 32 keys
+  // this CTA's range; thread t owns its elements [t E, t E + E)
   const int per = (m_total + csize - 1) / csize;
   const int c0 = min(m_total, per * rank), c1 = min(m_total, c0 + per);
-  const int wbase = c0 + warp * (E * 32);
+  const int n_cta = c1 - c0;
+  const int n_mine = max(0, min(E, n_cta - (int)threadIdx.x * E));  // valid keys of this thread
+#pragma unroll 8
+  for (int i = threadIdx.x; i < n_cta; i += kThreads)
+    big[(i / E) * Cfg::kPad + (i % E)] = keys[c0 + i];
+  __syncthreads();
   unsigned key[E];
 #pragma unroll
-  for (int i = 0; i < E; ++i) {
-    const int idx = wbase + i * 32 + lane;
-    key[i] = idx < c1 ? keys[idx] : 0u;
+  for (int j = 0; j < E; j += 4) {
+    const uint4 q = *reinterpret_cast<const uint4*>(&big[threadIdx.x * Cfg::kPad + j]);
+    key[j] = q.x;
+    key[j + 1] = q.y;
+    key[j + 2] = q.z;
+    key[j + 3] = q.w;
   }
+  __syncthreads();
+  for (int i = threadIdx.x; i < Cfg::kHistWords / 4; i += kThreads)
+    reinterpret_cast<uint4*>(big)[i] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
 
   // ---- radix passes: find tau and the number of ties to take -------------------------------
   unsigned prefix_val = 0, prefix_mask = 0;
@@ -248,30 +278,48 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
   if (k_sel > 0) {
     const int shifts[3] = {21, 10, 0};
     const int widths[3] = {11, 11, 10};
+    unsigned* my_copy = big + (lane & (Cfg::kRep - 1));
 #pragma unroll 1
     for (int pass = 0; pass < 3; ++pass) {
       const int shift = shifts[pass];
       const unsigned dmask = (1u << widths[pass]) - 1u;
-      for (int i = threadIdx.x; i < kBins; i += kThreads) sh.hist[i] = 0;
-      __syncthreads();
 #pragma unroll
-      for (int i = 0; i < E; ++i) {
-        const bool mine = wbase + i * 32 + lane < c1 && (key[i] & prefix_mask) == prefix_val;
-        const unsigned digit = (key[i] >> shift) & dmask;
-        // one shared-memory atomic per distinct digit in the warp
-        const unsigned active = __ballot_sync(0xffffffffu, mine);
-        if (mine) {
-          const unsigned peers = __match_any_sync(active, digit);
-          if (lane == (__ffs(peers) - 1)) atomicAdd(&sh.hist[digit], (unsigned)__popc(peers));
-        }
+      for (int j = 0; j < E; ++j) {
+        const unsigned digit = (key[j] >> shift) & dmask;
+        if (j < n_mine && (key[j] & prefix_mask) == prefix_val)
+          atomicAdd(&my_copy[digit * Cfg::kRep], 1u);
+      }
+      __syncthreads();
+      // Fold the copies and clear them: consecutive lanes take consecutive 16-byte pieces
+      // (conflict-free); kRep / 4 neighbouring lanes hold the pieces of one bin.
+      for (int i = threadIdx.x; i < Cfg::kHistWords / 4; i += kThreads) {
+        uint4* cell = reinterpret_cast<uint4*>(big) + i;
+        const uint4 q = *cell;
+        *cell = make_uint4(0u, 0u, 0u, 0u);
+        unsigned sum = q.x + q.y + q.z + q.w;
+#pragma unroll
+        for (int o = 1; o < Cfg::kRep / 4; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if ((i & (Cfg::kRep / 4 - 1)) == 0) sh.hist[i / (Cfg::kRep / 4)] = sum;
       }
       cluster.sync();  // every CTA's histogram is complete
-      for (int i = threadIdx.x; i < kBins; i += kThreads) {
-        unsigned sum = 0;
-        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(sh.hist, r)[i];
-        sh.total[i] = sum;
+      // CTA r sums bins [r * kBins / csize, ...) over the cluster and hands the sums to every
+      // CTA: each thread issues independent remote loads, then csize remote stores.
+      {
+        const int share = kBins / csize;  // 256 or 128
+        if ((int)threadIdx.x < share) {
+          const int bin = rank * share + threadIdx.x;
+          unsigned sum = 0;
+          for (int r0 = 0; r0 < csize; r0 += 8) {  // cluster sizes are 8 and 16
+            unsigned part[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) part[r] = cluster.map_shared_rank(sh.hist, r0 + r)[bin];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) sum += part[r];
+          }
+          for (int r = 0; r < csize; ++r) cluster.map_shared_rank(sh.total, r)[bin] = sum;
+        }
       }
-      cluster.sync();  // peers have finished reading this CTA's histogram
+      cluster.sync();  // all sums have arrived; peers have finished reading this CTA's histogram
       // Walk the digits from the top: thread t owns digits [kBins-1-4t-3, kBins-1-4t].
       unsigned mine4[4], local = 0;
 #pragma unroll
@@ -299,74 +347,76 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
   const unsigned tau = k_sel > 0 ? prefix_val : 0xffffffffu;
   const unsigned ties_wanted = k_sel > 0 ? (unsigned)k_rem : 0u;  // >= 1 when k_sel > 0
 
-  // ---- counts per warp, then the number of kept entries / ties before this warp ---------------
+  // ---- counts: per thread, then block scan (both counts packed, each at most 32768) ----------
   unsigned n_gt = 0, n_eq = 0;
 #pragma unroll
-  for (int i = 0; i < E; ++i) {
-    const bool valid = wbase + i * 32 + lane < c1;
-    n_gt += __popc(__ballot_sync(0xffffffffu, valid && key[i] > tau));
-    n_eq += __popc(__ballot_sync(0xffffffffu, valid && key[i] == tau));
+  for (int j = 0; j < E; ++j) {
+    n_gt += (j < n_mine && key[j] > tau) ? 1u : 0u;
+    n_eq += (j < n_mine && key[j] == tau) ? 1u : 0u;
   }
-  if (lane == 0) sh.warp_cnt[warp] = make_uint2(n_gt, n_eq);
+  unsigned cta_packed;
+  const unsigned before_packed = block_exclusive_scan(n_gt | (n_eq << 16), sh.warp_sum, &cta_packed);
+  const unsigned gt_before = before_packed & 0xffffu, eq_before = before_packed >> 16;
+  const unsigned cta_gt = cta_packed & 0xffffu, cta_eq = cta_packed >> 16;
+  if (threadIdx.x == 0) sh.cta_cnt = make_uint2(cta_gt, cta_eq);
   cluster.sync();
-  // warps in element order: (CTA rank, warp); lane l folds entries l, l + 32, ...
-  unsigned kept_base = 0, tie_base = 0;
-  {
-    const int mine = rank * kWarps + warp;  // entries before this warp
-    // ties are taken in order, so the kept count needs a sequential fold over the tie counts;
-    // lanes first add up the "above" counts and the ties of their entries, in order
-    unsigned gt_sum = 0, eq_sum = 0;
-    for (int e = lane; e < mine; e += 32) {
-      const uint2 c = cluster.map_shared_rank(sh.warp_cnt, e / kWarps)[e % kWarps];
-      gt_sum += c.x;
-      eq_sum += c.y;
-    }
+  unsigned gt_cta_before = 0, eq_cta_before = 0;  // counts in the CTAs before this one
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      gt_sum += __shfl_xor_sync(0xffffffffu, gt_sum, o);
-      eq_sum += __shfl_xor_sync(0xffffffffu, eq_sum, o);
+  for (int r = 0; r < 16; ++r)
+    if (r < rank) {
+      const uint2 c = *cluster.map_shared_rank(&sh.cta_cnt, r);
+      gt_cta_before += c.x;
+      eq_cta_before += c.y;
     }
-    tie_base = eq_sum;                                   // ties in earlier warps
-    kept_base = gt_sum + min(eq_sum, ties_wanted);       // the earliest ties are the ones taken
-  }
-  cluster.sync();  // counts stay valid until every CTA has read them
+  // ties are taken in element order: the earliest ties_wanted of them
+  const unsigned ties_before_cta = min(eq_cta_before, ties_wanted);
+  const unsigned kept_cta_before = gt_cta_before + ties_before_cta;
+  const unsigned cta_kept = cta_gt + (min(eq_cta_before + cta_eq, ties_wanted) - ties_before_cta);
 
-  // ---- ordered emit ------------------------------------------------------------------------------
-  int head = 0, pos = 0;
-  if (s.prefix > 0) {
-    const int first = wbase + lane;
-    head = first / s.prefix;
-    pos = first - head * s.prefix;
-  }
-  unsigned kept_run = kept_base, tie_run = tie_base;
+  // ---- ordered emit: pack the kept positions in shared memory, then store them coalesced -----
+  {
+    const unsigned tie0 = eq_cta_before + eq_before;  // index of this thread's first tie
+    const unsigned slot0 = gt_before + (min(tie0, ties_wanted) - ties_before_cta);  // in the CTA
+    // bit j of keep_mask: key j is retained (above tau, or one of the first ties_wanted ties)
+    unsigned long long keep_mask = 0ull;
+    {
+      unsigned ties_seen = 0;
 #pragma unroll
-  for (int i = 0; i < E; ++i) {
-    const int idx = wbase + i * 32 + lane;
-    const bool valid = idx < c1;
-    const bool gt = valid && key[i] > tau, eq = valid && key[i] == tau;
-    const unsigned eq_mask = __ballot_sync(0xffffffffu, eq);
-    const unsigned lt = (1u << lane) - 1u;
-    const bool keep = gt || (eq && tie_run + __popc(eq_mask & lt) < ties_wanted);
-    const unsigned keep_mask = __ballot_sync(0xffffffffu, keep);
-    const unsigned my_slot = kept_run + __popc(keep_mask & lt);
-    if (valid) {
-      if (keep) out[my_slot] = pos;
-      // the first entry of a head records how many kept entries precede the head
-      if (pos == 0) hoff[head] = (int)my_slot + head * g.window;
+      for (int j = 0; j < E; ++j) {
+        const bool eq = j < n_mine && key[j] == tau;
+        const bool keep = (j < n_mine && key[j] > tau) || (eq && tie0 + ties_seen < ties_wanted);
+        keep_mask |= (unsigned long long)keep << j;
+        ties_seen += eq ? 1u : 0u;
+      }
     }
-    kept_run += __popc(keep_mask);
-    tie_run += __popc(eq_mask);
-    pos += 32;
-    while (s.prefix > 0 && pos >= s.prefix) {
-      pos -= s.prefix;
-      ++head;
+    int* packed = reinterpret_cast<int*>(big);
+    if (n_mine > 0) {
+      const int first = c0 + (int)threadIdx.x * E;
+      int head = first / s.prefix;
+      const int pos0 = first - head * s.prefix;
+      // heads that start inside this thread's keys record how many kept entries precede them
+      for (int j = pos0 == 0 ? 0 : s.prefix - pos0; j < n_mine; j += s.prefix) {
+        const int h = (first + j) / s.prefix;
+        hoff[h] = (int)(kept_cta_before + slot0) + __popcll(keep_mask & ((1ull << j) - 1ull)) +
+                  h * g.window;
+      }
+#pragma unroll
+      for (int j = 0; j < E; ++j) {
+        int pos = pos0 + j;
+        while (pos >= s.prefix) pos -= s.prefix;  // at most once unless heads are shorter than E
+        if ((keep_mask >> j) & 1ull)
+          packed[slot0 + __popcll(keep_mask & ((1ull << j) - 1ull))] = pos;
+      }
     }
+    __syncthreads();
+    for (unsigned i = threadIdx.x; i < cta_kept; i += kThreads) out[kept_cta_before + i] = packed[i];
   }
   if (rank == 0 && threadIdx.x == 0) {
     hoff[g.n_kv_heads] = (int)(k_sel + window_rows);
     if (s.prefix == 0)  // no candidates: every head holds only its (possibly short) window
       for (int h = 0; h < g.n_kv_heads; ++h) hoff[h] = h * min(g.window, s.n);
   }
+  cluster.sync();  // peers may still be reading this CTA's counts
 }
 
 template <int E>
@@ -374,6 +424,11 @@ cudaError_t launch_reg(const Geom& g, int problems, int csize, const float* scor
                        const long long* layer_budget, int* keep_idx, int* head_offsets,
                        cudaStream_t stream) {
   auto kern = select_topk_reg_kernel<E>;
+  const int big_bytes = RegCfg<E>::kBigWords * (int)sizeof(unsigned);
+  {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, big_bytes);
+    if (e != cudaSuccess) return e;
+  }
   if (csize > 8) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
@@ -381,6 +436,7 @@ cudaError_t launch_reg(const Geom& g, int problems, int csize, const float* scor
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(csize * problems);
   cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = big_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeClusterDimension;
