@@ -221,6 +221,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2509_09754_b200 as lava
+    from paper_2509_09754_b200 import replicas
     from lava_workloads import generate_layer, get_config
 
     if not torch.cuda.is_available():
@@ -304,15 +305,11 @@ def main():
     if world > 1:
         dist.barrier()
     launches = lava.lava_launch_count() - launches0
-    total_ms = t_start.elapsed_time(t_end)
-    if world > 1:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = replicas.slowest_rank_ms(t_start.elapsed_time(t_end))
     ms_per_step = total_ms / steps
     phase_ms = [sum(ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(steps)) / steps
                 for j in range(4)]
-    value = world * cfg.total_tokens / (ms_per_step * 1e-3)
+    value = replicas.whole_job_units(cfg.total_tokens) / (ms_per_step * 1e-3)
 
     kv_bytes, out_bytes = roofline_bytes(cfg)
     peak, peak_src = measured_hbm_peak()
