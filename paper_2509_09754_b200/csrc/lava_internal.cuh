@@ -69,6 +69,7 @@ lava_status launch_score_generic(const Geom& g, int n_layers, const void* q, con
 // Blackwell tensor-core score path (bf16, head_dim 128, G*w <= 128).
 struct Sm100Layout {
   int heads_total, chunks1, chunks2, out_keys;  // chunks per head at max_seqlen, pass 1 / pass 2
+  int chunk_tiles;                              // tiles per chunk chosen for this launch
   size_t off_sync, sync_bytes, off_part, off_ent, total;
 };
 bool sm100_supported(const Geom& g);

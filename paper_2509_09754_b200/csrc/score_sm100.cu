@@ -429,14 +429,14 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     mbar_init(smem_u32(&m->q2_empty), 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&m->s1_full[s]), 1);
-      mbar_init(smem_u32(&m->s1_empty[s]), 128);
+      mbar_init(smem_u32(&m->s1_empty[s]), 4);   // one arrival per warp of the group
       mbar_init(smem_u32(&m->s2_full[s]), 1);
-      mbar_init(smem_u32(&m->s2_empty[s]), 128);
-      mbar_init(smem_u32(&m->pub_full[s]), 256);
+      mbar_init(smem_u32(&m->s2_empty[s]), 4);
+      mbar_init(smem_u32(&m->pub_full[s]), 8);   // the eight consumer warps
       mbar_init(smem_u32(&m->pub_empty[s]), 1);
       mbar_init(smem_u32(&m->prep_full[s]), 1);
       mbar_init(smem_u32(&m->prep_empty[s]), 8);
-      mbar_init(smem_u32(&m->gsync[s]), 128);
+      mbar_init(smem_u32(&m->gsync[s]), 4);
     }
     mbar_init(smem_u32(&m->drain), 1);
     mbar_init(smem_u32(&m->drain2), 1);
@@ -732,7 +732,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     bool alive = true;
     // rendezvous of the group's four warps (bounded, and it ends when the CTA aborts)
     auto group_sync = [&]() {
-      mbar_arrive(gbar);
+      __syncwarp();  // the lanes' shared-memory writes are ordered before lane 0's arrival
+      if (lane == 0) mbar_arrive(gbar);
       if (!__all_sync(0xffffffffu, wait_bar(gbar, gphase & 1, m, p.status))) alive = false;
       ++gphase;
     };
@@ -768,7 +769,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
             break;
           }
           m->pub[slot][grp][row] = z > 0.f ? mx + fast_log2(z) : -INFINITY;
-          mbar_arrive(smem_u32(&m->pub_full[slot]));
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&m->pub_full[slot]));
           mx = -INFINITY;
           z = 0.f;
           ++j1;
@@ -876,7 +878,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           }
         }
         tc_fence_before();
-        mbar_arrive(smem_u32(&m->s1_empty[grp]));
+        __syncwarp();  // every lane has finished reading the accumulator
+        if (lane == 0) mbar_arrive(smem_u32(&m->s1_empty[grp]));
         ++t1;
         ++n1;
       } else {
@@ -941,7 +944,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           }
         }
         tc_fence_before();
-        mbar_arrive(smem_u32(&m->s2_empty[grp]));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&m->s2_empty[grp]));
         // lane <-> key: the tile starts pool_radius keys before the first key it owns; keys
         // outside the prefix hold the neutral element of both pools (values are >= 0)
         const int ab = (int)((n2 >> 1) & 1);
@@ -1164,28 +1168,36 @@ EncodeTiledFn encode_fn() {
 
 size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
-// tiles per chunk: tuning knob (LAVA_SM100_CHUNK_TILES), default 8
-int chunk_tiles_setting() {
-  static int value = 0;
-  if (!value) {
+// Tiles per chunk.  A chunk boundary costs a reload of the head's query tile and a hand-over
+// of statistics, so chunks should be long; but the launch needs many more chunks than CTAs to
+// balance (chunks are dealt round-robin), and a head finishes pass 1 sooner when more CTAs
+// share it.  Default: about twelve chunks per CTA, between 4 and 32 tiles.  LAVA_SM100_CHUNK_TILES
+// overrides it.
+constexpr int kMinChunkTiles = 4, kMaxChunkTiles = 32;
+int chunk_tiles_for(const Geom& g, int n_layers) {
+  static int forced = -1;
+  if (forced < 0) {
     const char* e = getenv("LAVA_SM100_CHUNK_TILES");
     const int v = e ? atoi(e) : 0;
-    value = (v >= 1 && v <= 64) ? v : 8;
+    forced = (v >= 1 && v <= 64) ? v : 0;
   }
-  return value;
+  if (forced) return forced;
+  const long long tiles = (long long)n_layers * g.n_kv_heads * ceil_div((int)g.total_tokens, kTile);
+  const long long r = tiles / (148 * 12);
+  return (int)(r < kMinChunkTiles ? kMinChunkTiles : r > kMaxChunkTiles ? kMaxChunkTiles : r);
 }
 
-
-// tiles pass 1 leads pass 2 by beyond what head completion needs (covers the time a head's
-// statistics take to be published and folded): tuning knob (LAVA_SM100_LEAD_TILES), default 3
-int lead_extra_setting() {
-  static int value = -1;
-  if (value < 0) {
+// Tiles pass 1 leads pass 2 by beyond what head completion needs (covers the time a head's
+// statistics take to be published and folded, and the skew between CTAs): half a chunk.
+// LAVA_SM100_LEAD_TILES overrides it.
+int lead_extra_for(int chunk_tiles) {
+  static int forced = -2;
+  if (forced == -2) {
     const char* e = getenv("LAVA_SM100_LEAD_TILES");
     const int v = e ? atoi(e) : -1;
-    value = (v >= 0 && v <= 4096) ? v : 3;
+    forced = (v >= 0 && v <= 4096) ? v : -1;
   }
-  return value;
+  return forced >= 0 ? forced : (chunk_tiles + 1) / 2;
 }
 
 }  // namespace
@@ -1202,11 +1214,14 @@ bool sm100_supported(const Geom& g) {
 
 Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   Sm100Layout l;
-  const int r = chunk_tiles_setting();
+  const int r = chunk_tiles_for(g, n_layers);
+  l.chunk_tiles = r;
   l.heads_total = n_layers * g.batch * g.n_kv_heads;
   l.out_keys = kTile - 2 * g.pool_radius;
-  l.chunks1 = ceil_div(ceil_div(g.max_seqlen, kTile), r);                       // chunks, pass 1
-  l.chunks2 = ceil_div(ceil_div(max(1, g.max_seqlen - g.window), l.out_keys), r);  // chunks, pass 2
+  const int tiles1 = ceil_div(g.max_seqlen, kTile);
+  const int tiles2 = ceil_div(max(1, g.max_seqlen - g.window), l.out_keys);
+  l.chunks1 = ceil_div(tiles1, r);  // chunks per head, pass 1
+  l.chunks2 = ceil_div(tiles2, r);  // chunks per head, pass 2
   size_t off = 0;
   l.off_sync = off;   // chunk counters, value-norm counters and bits: zeroed every launch
   off = up256(off + sizeof(int) * 3 * (size_t)l.heads_total);
@@ -1215,7 +1230,14 @@ Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   off = up256(off + sizeof(float) * 128 * (size_t)l.heads_total * l.chunks1);
   l.off_ent = off;
   off = up256(off + sizeof(float2) * 8 * (size_t)l.heads_total * l.chunks2);
-  l.total = off;
+  // The size asked of the caller does not depend on the chunk length chosen for this launch
+  // (a workspace sized for a whole model also serves calls on fewer layers): it is the size
+  // at the shortest chunk.
+  const int rmin = r < kMinChunkTiles ? r : kMinChunkTiles;
+  size_t cap = up256(sizeof(int) * 3 * (size_t)l.heads_total);
+  cap = up256(cap + sizeof(float) * 128 * (size_t)l.heads_total * ceil_div(tiles1, rmin));
+  cap = up256(cap + sizeof(float2) * 8 * (size_t)l.heads_total * ceil_div(tiles2, rmin));
+  l.total = cap > off ? cap : off;
   return l;
 }
 
@@ -1264,11 +1286,11 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   Sm100Params p;
   p.g = g;
   p.n_layers = n_layers;
-  p.chunk_tiles = chunk_tiles_setting();
+  p.chunk_tiles = lay.chunk_tiles;
   p.out_keys = lay.out_keys;
   p.cph1_max = lay.chunks1;
   p.cph2_max = lay.chunks2;
-  p.lead_extra = lead_extra_setting();
+  p.lead_extra = lead_extra_for(lay.chunk_tiles);
   p.vbar_in = vbar_in;
   p.scores = scores;
   p.vbar_out = vbar_out;
