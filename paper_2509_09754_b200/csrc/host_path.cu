@@ -32,7 +32,8 @@ Arena arena_layout(const lava_layer_desc* d, int n_layers, long long rows) {
   const size_t total_scores =
       (size_t)d->n_kv_heads * (size_t)(d->total_tokens - (long long)d->batch * d->window);
   lava_layer_desc one = *d;
-  one.cu_seqlens = nullptr;
+  // sizes do not read the offsets; batches need a non-null pointer to pass validation
+  one.cu_seqlens = d->batch > 1 ? reinterpret_cast<const int32_t*>(16) : nullptr;
   a.ws_bytes = workspace_layout(&one, 1).total;
   a.q_layer = (size_t)d->batch * d->n_q_heads * d->window * d->head_dim * es;
   a.kv_layer = (size_t)d->n_kv_heads * d->total_tokens * d->head_dim * es;

@@ -90,6 +90,8 @@ struct Sm100Params {
   int out_keys;             // keys a pass-2 tile owns: 128 - 2 * pool_radius
   int cph1_max, cph2_max;   // chunks per head at max_seqlen (strides of the scratch arrays)
   int lead_extra;           // tiles pass 1 leads pass 2 by, beyond what head completion needs
+  int split;                // 1: every KV head is scored as two halves of its query group
+  int g0;                   // query heads in the first half (split mode)
   const float* vbar_in;
   float* scores;
   float* vbar_out;
@@ -308,8 +310,13 @@ __device__ inline bool wait_bar(uint32_t bar, uint32_t parity, Misc* m, unsigned
 // chunk schedule (identical in every role and every CTA, so no descriptors travel)
 // ------------------------------------------------------------------------------------------
 struct Chunk {
-  int head;    // linear head index = (layer * batch + b) * H_kv + kvh
+  int head;    // linear index of the scored unit (a KV head, or one half of its query group in
+               // split mode): counters, chunk partials and entropy slots are per unit
+  int rhead;   // linear KV head index = (layer * batch + b) * H_kv + kvh (value norms)
   int layer, b, kvh;
+  int half;    // which half of the query group (0 unless split)
+  int q0;      // first query head of the unit inside the sequence's H_q heads
+  int group;   // query heads of the unit
   int index;   // chunk number inside the head
   int cph;     // chunks of this head
   int tile0, ntiles;
@@ -326,7 +333,7 @@ __device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, int c,
   Chunk ck;
   ck.layer = c / per_layer;
   const int r = c - ck.layer * per_layer;
-  const int hkv = p.g.n_kv_heads;
+  const int hkv = p.g.n_kv_heads << p.split;  // scored units per sequence
   int lo = 0, hi = p.g.batch;  // largest b with hkv * pref[b] <= r
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
@@ -335,9 +342,14 @@ __device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, int c,
   ck.b = lo;
   ck.cph = pref[lo + 1] - pref[lo];
   const int r2 = r - hkv * pref[lo];
-  ck.kvh = r2 / ck.cph;
-  ck.index = r2 - ck.kvh * ck.cph;
-  ck.head = (ck.layer * p.g.batch + ck.b) * hkv + ck.kvh;
+  const int unit = r2 / ck.cph;
+  ck.index = r2 - unit * ck.cph;
+  ck.head = (ck.layer * p.g.batch + ck.b) * hkv + unit;
+  ck.half = p.split ? (unit & 1) : 0;
+  ck.kvh = unit >> p.split;
+  ck.rhead = (ck.layer * p.g.batch + ck.b) * p.g.n_kv_heads + ck.kvh;
+  ck.group = p.split ? (ck.half ? p.g.group - p.g0 : p.g0) : p.g.group;
+  ck.q0 = ck.kvh * p.g.group + ck.half * p.g0;
   ck.s = seq_info(p.g, ck.b);
   ck.tile0 = ck.index * p.chunk_tiles;
   ck.ntiles = min(p.chunk_tiles, tiles_of(p, ck.s, pass) - ck.tile0);
@@ -357,7 +369,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
   Misc* m = reinterpret_cast<Misc*>(gen + kOffMisc);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Geom& g = p.g;
-  const int rows_valid = g.group * W;
+  const int units = g.n_kv_heads << p.split;  // scored units per sequence
 
   // ---- chunk schedule: exclusive scans of chunks per sequence, both passes -------------------
   {
@@ -397,8 +409,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-      m->sched_total1 = g.n_kv_heads * m->pref1[g.batch];
-      m->sched_total2 = g.n_kv_heads * m->pref2[g.batch];
+      m->sched_total1 = units * m->pref1[g.batch];
+      m->sched_total2 = units * m->pref2[g.batch];
       // How far pass 1 must lead pass 2 in a CTA's own order (see the consumer warps).  With
       // rho = pass-2 chunks per pass-1 chunk: rho * (1 + (longest head + drift) / grid) chunks,
       // where drift is how far the two passes' chunk numbering can diverge inside a layer.
@@ -407,8 +419,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       double drift = 0.0, longest = 0.0;
       for (int b = 0; b < g.batch; ++b) {
         const double c1 = m->pref1[b + 1] - m->pref1[b], c2 = m->pref2[b + 1] - m->pref2[b];
-        const double at = fabs(g.n_kv_heads * (m->pref1[b] * rho - m->pref2[b]));
-        drift = fmax(drift, at + g.n_kv_heads * fabs(c1 * rho - c2));
+        const double at = fabs(units * (m->pref1[b] * rho - m->pref2[b]));
+        drift = fmax(drift, at + units * fabs(c1 * rho - c2));
         longest = fmax(longest, c1);
       }
       const double lead = p.chunk_tiles * rho * (1.0 + (longest + drift) / (double)gridDim.x);
@@ -471,7 +483,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         {
           const uint32_t bar = smem_u32(&m->q1_full);
           mbar_expect_tx(bar, kTileBytes);
-          const int row0 = (ck.b * g.n_q_heads + ck.kvh * g.group) * W;
+          const int row0 = (ck.b * g.n_q_heads + ck.q0) * W;
           tma_load_3d(base + kOffQ1, &map_q, 0, row0, ck.layer, bar);
           tma_load_3d(base + kOffQ1 + kHalfBytes, &map_q, 64, row0, ck.layer, bar);
           ++q_loads;
@@ -513,7 +525,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         const int want_v = p.vbar_in ? 0 : kVWarps * cph1;
         const long long t0 = clock64();
         while (ld_acquire(&p.counters[ck.head]) < cph1 ||
-               (want_v && ld_acquire(&p.vcount[ck.head]) < want_v)) {
+               (want_v && ld_acquire(&p.vcount[ck.rhead]) < want_v)) {
           if (m->abort_flag) break;
           __nanosleep(100);
           if (clock64() - t0 > kWaitCycles) give_up(m, p.status);
@@ -581,8 +593,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       if (lane == 0) {
-        const float vb = p.vbar_in ? p.vbar_in[ck.head]
-                                   : __uint_as_float(__ldcg(p.vbar_bits + ck.head));
+        const float vb = p.vbar_in ? p.vbar_in[ck.rhead]
+                                   : __uint_as_float(__ldcg(p.vbar_bits + ck.rhead));
         m->prep[slot].scale = vb * g.c_hat;
       }
       __syncwarp();
@@ -592,7 +604,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         if (ok) {
           const uint32_t bar = smem_u32(&m->q2_full);
           mbar_expect_tx(bar, kTileBytes);
-          const int row0 = (ck.b * g.n_q_heads + ck.kvh * g.group) * W;
+          const int row0 = (ck.b * g.n_q_heads + ck.q0) * W;
           tma_load_3d(base + kOffQ2, &map_q, 0, row0, ck.layer, bar);
           tma_load_3d(base + kOffQ2 + kHalfBytes, &map_q, 64, row0, ck.layer, bar);
           ++q_loads;
@@ -726,7 +738,6 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     const float inv_w = 1.0f / (float)W;
     const float sc2 = g.scale_log2;
     const bool avg = g.pool_kind == LAVA_POOL_AVG;
-    const int nblk = (rows_valid + 31) >> 5;  // 32-column blocks of window queries in use
     const uint32_t gbar = smem_u32(&m->gsync[grp]);
     uint32_t gphase = 0;
     bool alive = true;
@@ -747,7 +758,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     auto open1 = [&]() {
       k1 = decode_chunk(p, m, c1, 1);
       // keys this query may see: i < n and i <= P + t
-      last1 = row < rows_valid ? min(k1.s.n, k1.s.prefix + t_in_win + 1) : 0;
+      last1 = row < k1.group * W ? min(k1.s.n, k1.s.prefix + t_in_win + 1) : 0;
     };
     if (has1) open1();
     int c2 = blockIdx.x, t2 = 0;
@@ -902,6 +913,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + 256u + (uint32_t)grp * 128u;
         // window queries come in blocks of 32 columns; a block lies inside one query head when
         // W >= 32, and holds two heads when W == 16
+        const int nblk = (k2.group * W + 31) >> 5;  // 32-column blocks of window queries in use
 #pragma unroll 1
         for (int blk = 0; blk < nblk; ++blk) {
           float cur[32];
@@ -955,13 +967,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         if (avg) {
 #pragma unroll
           for (int h = 0; h < NH; ++h)
-            if (h < 4 && h < g.group) abuf[h][row] = inside ? acc[h] * inv_w : 0.f;
+            if (h < 4 && h < k2.group) abuf[h][row] = inside ? acc[h] * inv_w : 0.f;
         } else {
           // max-pooling commutes with the group maximum: reduce over the query heads first
           float top = 0.f;
 #pragma unroll
           for (int h = 0; h < NH; ++h)
-            if (h < g.group) top = fmaxf(top, acc[h] * inv_w);
+            if (h < k2.group) top = fmaxf(top, acc[h] * inv_w);
           abuf[0][row] = inside ? top : 0.f;
         }
         group_sync();
@@ -970,7 +982,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         if (i >= own_lo && i < own_hi) {
           float best = 0.f;
           if (avg) {
-            for (int h = 0; h < g.group; ++h) {
+            for (int h = 0; h < k2.group; ++h) {
               const float* a = &abuf[h][row];
               float pv = 0.f;
               for (int q = -rad; q <= rad; ++q) pv += a[q];
@@ -987,8 +999,12 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
             }
           }
           const float sc = best * prep->scale;
-          p.scores[(size_t)k2.layer * g.total_scores + k2.s.score_off +
-                   (long long)k2.kvh * k2.s.prefix + i] = sc;
+          float* dst = p.scores + (size_t)k2.layer * g.total_scores + k2.s.score_off +
+                       (long long)k2.kvh * k2.s.prefix + i;
+          // split mode: the group maximum over the two halves is taken in memory (scores are
+          // >= 0, so their bit patterns order like the values; the array starts as zeros)
+          if (p.split) atomicMax(reinterpret_cast<unsigned*>(dst), __float_as_uint(sc));
+          else *dst = sc;
           if (sc > 0.f) {
             es += sc;
             et += sc * __logf(sc);
@@ -1026,12 +1042,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           c += gridDim.x;
           grp = 0;
           ngrp = ceil_div(min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile) - ck.tile0 * kTile, 8 * kVRows);
+          if (ck.half) ngrp = 0;  // the head's V rows belong to the first half's chunks
         }
         gr.base = p.v + ((size_t)ck.layer * p.v_ls + (long long)ck.kvh * g.v_sh +
                          ck.s.tok0 * g.v_st) * 2 + tq * 16;
         gr.row0 = ck.tile0 * kTile + grp * 8 * kVRows + vw * 16 + gq;
         gr.row_hi = min(ck.s.n, (ck.tile0 + ck.ntiles) * kTile);
-        gr.head = ck.head;
+        gr.head = ck.rhead;
         gr.last = ++grp == ngrp;
         return true;
       };
@@ -1145,6 +1162,57 @@ entropy_finalize_sm100_kernel(Geom g, const float2* ent_part, int cph2_max, int 
   }
 }
 
+// Split mode: the scores of a KV head are complete only after both halves of its query group
+// have been merged in memory, so the entropy of one (layer, sequence) is summed from the final
+// score array here (fixed order: thread-strided fp32 sums of at most a few hundred terms, then
+// fp64 across lanes and warps).  Also hands out the value norms.
+__global__ void __launch_bounds__(1024)
+entropy_from_scores_kernel(Geom g, const float* scores, double* entropy, const float* vbar_in,
+                           const unsigned* vbar_bits, float* vbar_out) {
+  __shared__ double rs[32], rt[32];
+  const int prob = blockIdx.x, layer = prob / g.batch, b = prob - layer * g.batch;
+  const SeqInfo s = seq_info(g, b);
+  if (vbar_out && (int)threadIdx.x < g.n_kv_heads) {
+    const size_t head = (size_t)prob * g.n_kv_heads + threadIdx.x;
+    vbar_out[head] = vbar_in ? vbar_in[head] : __uint_as_float(vbar_bits[head]);
+  }
+  const float* sc = scores + (size_t)layer * g.total_scores + s.score_off;
+  const long long count = (long long)g.n_kv_heads * s.prefix;
+  double sum_s = 0.0, sum_t = 0.0;
+  for (long long i0 = threadIdx.x; i0 < count; i0 += 1024 * 256) {
+    float es = 0.f, et = 0.f;  // at most 256 terms in fp32, then fp64
+    for (long long i = i0; i < count && i < i0 + 1024LL * 256; i += 1024) {
+      const float v = sc[i];
+      if (v > 0.f) {
+        es += v;
+        et += v * __logf(v);
+      }
+    }
+    sum_s += (double)es;
+    sum_t += (double)et;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    sum_s += __shfl_down_sync(0xffffffffu, sum_s, o);
+    sum_t += __shfl_down_sync(0xffffffffu, sum_t, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    rs[threadIdx.x >> 5] = sum_s;
+    rt[threadIdx.x >> 5] = sum_t;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0.0, c = 0.0;
+    for (int i = 0; i < 32; ++i) {
+      a += rs[i];
+      c += rt[i];
+    }
+    double e = 0.0;
+    if (a > 0.0) e = (log(a) - c / a) / ((double)g.n_kv_heads * (double)s.n);
+    entropy[(size_t)layer * g.batch + b] = e;
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------
@@ -1174,6 +1242,13 @@ size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 // share it.  Default: about twelve chunks per CTA, between 4 and 32 tiles.  LAVA_SM100_CHUNK_TILES
 // overrides it.
 constexpr int kMinChunkTiles = 4, kMaxChunkTiles = 32;
+
+// Query groups of more than 128 window-query rows are scored as two halves (each a unit of its
+// own with at most 128 rows); returns the number of query heads in the first half, 0 if the
+// group fits one unit.
+int sm100_first_half(const Geom& g) {
+  return g.group * g.window > 128 ? (g.group + 1) / 2 : 0;
+}
 int chunk_tiles_for(const Geom& g, int n_layers) {
   static int forced = -1;
   if (forced < 0) {
@@ -1182,7 +1257,8 @@ int chunk_tiles_for(const Geom& g, int n_layers) {
     forced = (v >= 1 && v <= 64) ? v : 0;
   }
   if (forced) return forced;
-  const long long tiles = (long long)n_layers * g.n_kv_heads * ceil_div((int)g.total_tokens, kTile);
+  const long long tiles = (long long)n_layers * (g.n_kv_heads << (sm100_first_half(g) ? 1 : 0)) *
+                          ceil_div((int)g.total_tokens, kTile);
   const long long r = tiles / (148 * 12);
   return (int)(r < kMinChunkTiles ? kMinChunkTiles : r > kMaxChunkTiles ? kMaxChunkTiles : r);
 }
@@ -1205,8 +1281,11 @@ int lead_extra_for(int chunk_tiles) {
 bool sm100_supported(const Geom& g) {
   if (g.dtype != LAVA_BF16 || g.head_dim != 128) return false;
   if (g.window != 16 && g.window != 32 && g.window != 64 && g.window != 128) return false;
-  if (g.group * g.window > 128 || g.group > 8) return false;
-  if (g.pool_kind == LAVA_POOL_AVG && g.group > 4) return false;  // room for 4 heads' window means
+  // heads of one scored unit: the whole query group, or its larger half when the group has more
+  // than 128 window-query rows
+  const int unit = g.group * g.window > 128 ? (g.group + 1) / 2 : g.group;
+  if (unit * g.window > 128 || unit > 8) return false;
+  if (g.pool_kind == LAVA_POOL_AVG && unit > 4) return false;  // room for 4 heads' window means
   if (g.pool_radius > 31) return false;
   if (g.batch > kMaxBatch) return false;
   return true;
@@ -1216,7 +1295,7 @@ Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   Sm100Layout l;
   const int r = chunk_tiles_for(g, n_layers);
   l.chunk_tiles = r;
-  l.heads_total = n_layers * g.batch * g.n_kv_heads;
+  l.heads_total = n_layers * g.batch * (g.n_kv_heads << (sm100_first_half(g) ? 1 : 0));  // units
   l.out_keys = kTile - 2 * g.pool_radius;
   const int tiles1 = ceil_div(g.max_seqlen, kTile);
   const int tiles2 = ceil_div(max(1, g.max_seqlen - g.window), l.out_keys);
@@ -1291,6 +1370,8 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.cph1_max = lay.chunks1;
   p.cph2_max = lay.chunks2;
   p.lead_extra = lead_extra_for(lay.chunk_tiles);
+  p.g0 = sm100_first_half(g);
+  p.split = p.g0 ? 1 : 0;
   p.vbar_in = vbar_in;
   p.scores = scores;
   p.vbar_out = vbar_out;
@@ -1306,6 +1387,11 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   rc = check_cuda(cudaMemsetAsync(ws + lay.off_sync, 0, lay.sync_bytes, stream),
                   "sync scratch clear");
   if (rc != LAVA_OK) return rc;
+  if (p.split) {  // the two halves of a query group meet in memory through a maximum
+    rc = check_cuda(cudaMemsetAsync(scores, 0, sizeof(float) * (size_t)n_layers * g.total_scores,
+                                    stream), "score clear");
+    if (rc != LAVA_OK) return rc;
+  }
 
   void (*kern)(const CUtensorMap, const CUtensorMap, const Sm100Params) = nullptr;
   switch (g.window) {
@@ -1327,9 +1413,13 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   rc = check_cuda(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args,
                                               kSmemBytes, stream), "score (sm100) launch");
   if (rc != LAVA_OK) return rc;
-  entropy_finalize_sm100_kernel<<<n_layers * g.batch, 256, 0, stream>>>(
-      g, p.ent_part, lay.chunks2, p.chunk_tiles * lay.out_keys, entropy, vbar_in, p.vbar_bits,
-      vbar_out);
+  if (p.split)
+    entropy_from_scores_kernel<<<n_layers * g.batch, 1024, 0, stream>>>(g, scores, entropy, vbar_in,
+                                                                        p.vbar_bits, vbar_out);
+  else
+    entropy_finalize_sm100_kernel<<<n_layers * g.batch, 256, 0, stream>>>(
+        g, p.ent_part, lay.chunks2, p.chunk_tiles * lay.out_keys, entropy, vbar_in, p.vbar_bits,
+        vbar_out);
   count_launches(2);
   return check_cuda(cudaGetLastError(), "entropy finalize launch");
 }
