@@ -221,6 +221,29 @@ __device__ inline float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Sum of 32 values by a fixed tree (i with i + 16, then + 8, + 4, then ((0 + 1) + (2 + 3))); the
+// wide levels use the packed two-lane fp32 add, which rounds each lane like the scalar add.
+__device__ inline float tree_sum32(float (&c)[32]) {
+#pragma unroll
+  for (int i = 0; i < 16; i += 2) {
+    const float2 r = __fadd2_rn(make_float2(c[i], c[i + 1]), make_float2(c[i + 16], c[i + 17]));
+    c[i] = r.x;
+    c[i + 1] = r.y;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; i += 2) {
+    const float2 r = __fadd2_rn(make_float2(c[i], c[i + 1]), make_float2(c[i + 8], c[i + 9]));
+    c[i] = r.x;
+    c[i + 1] = r.y;
+  }
+#pragma unroll
+  for (int i = 0; i < 4; i += 2) {
+    const float2 r = __fadd2_rn(make_float2(c[i], c[i + 1]), make_float2(c[i + 4], c[i + 5]));
+    c[i] = r.x;
+    c[i + 1] = r.y;
+  }
+  return (c[0] + c[1]) + (c[2] + c[3]);
+}
 __device__ inline float fast_log2(float x) {
   float y;
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -861,16 +884,15 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
             }
             const float neg = -mx;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) cur[i] = fmaf(cur[i], sc2, neg);
+            for (int i = 0; i < 32; i += 2) {
+              const float2 r = __ffma2_rn(make_float2(cur[i], cur[i + 1]), make_float2(sc2, sc2),
+                                          make_float2(neg, neg));
+              cur[i] = r.x;
+              cur[i + 1] = r.y;
+            }
 #pragma unroll
             for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i]);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) cur[i] += cur[i + 16];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) cur[i] += cur[i + 8];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) cur[i] += cur[i + 4];
-            z += (cur[0] + cur[1]) + (cur[2] + cur[3]);
+            z += tree_sum32(cur);
           } else if (cnt > 0) {
             float bm = -INFINITY;
 #pragma unroll
@@ -921,15 +943,13 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           tmem_ld_wait(cur);
           // the MMA has already subtracted the log-sum-exp: p = exp2(scale * logit)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) cur[i] = fast_exp2(cur[i] * sc2);
+          for (int i = 0; i < 32; i += 2) {
+            const float2 r = __fmul2_rn(make_float2(cur[i], cur[i + 1]), make_float2(sc2, sc2));
+            cur[i] = fast_exp2(r.x);
+            cur[i + 1] = fast_exp2(r.y);
+          }
           if (W >= 32) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) cur[i] += cur[i + 16];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) cur[i] += cur[i + 8];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) cur[i] += cur[i + 4];
-            const float sum = (cur[0] + cur[1]) + (cur[2] + cur[3]);
+            const float sum = tree_sum32(cur);
             const int h = (blk * 32) / W;
 #pragma unroll
             for (int hh = 0; hh < NH; ++hh)
