@@ -870,13 +870,15 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           tmem_ld_wait(cur);
           if (cnt >= 32) {
             // stage by stage (maxima, scaled differences, exponentials, a fixed summation tree)
-            float t[16];
+            // four running maxima (few live registers; the chains are independent)
+            float t[4] = {cur[0], cur[1], cur[2], cur[3]};
 #pragma unroll
-            for (int i = 0; i < 16; ++i) t[i] = fmaxf(cur[i], cur[i + 16]);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) t[i] = fmaxf(t[i], t[i + 8]);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) t[i] = fmaxf(t[i], t[i + 4]);
+            for (int i = 4; i < 32; i += 4) {
+              t[0] = fmaxf(t[0], cur[i]);
+              t[1] = fmaxf(t[1], cur[i + 1]);
+              t[2] = fmaxf(t[2], cur[i + 2]);
+              t[3] = fmaxf(t[3], cur[i + 3]);
+            }
             const float nm = fmaxf(fmaxf(t[0], t[1]), fmaxf(t[2], t[3])) * sc2;
             if (nm > mx) {
               z *= fast_exp2(mx - nm);
