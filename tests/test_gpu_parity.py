@@ -210,3 +210,20 @@ def test_host_buffer_path_equals_device_path():
         assert torch.equal(out_hoff, plan.head_offsets.cpu())
         assert torch.equal(out_k.view(torch.int16), plan.k_out.cpu().view(torch.int16))
         assert torch.equal(out_v.view(torch.int16), plan.v_out.cpu().view(torch.int16))
+
+@pytest.mark.parametrize("kw", [
+    # query groups of more than 128 window-query rows: two halves per KV head on the tensor-core path
+    dict(n_q_heads=8, n_kv_heads=2, window=64, seq_lens=(1500,)),                    # G 4 x w 64, max-pool
+    dict(n_q_heads=14, n_kv_heads=2, window=32, seq_lens=(1100, 700)),               # G 7: halves of 4 and 3
+    dict(n_q_heads=4, n_kv_heads=2, window=128, seq_lens=(1300,)),                   # G 2 x w 128: one head each
+    dict(n_q_heads=32, n_kv_heads=2, window=16, seq_lens=(900,)),                    # G 16 x w 16: 8 heads each
+    dict(n_q_heads=6, n_kv_heads=2, window=64, seq_lens=(1000,), pool_kind=lava.LAVA_POOL_AVG,
+         pool_kernel=5),                                                             # G 3: halves of 2 and 1, avg
+    dict(n_q_heads=8, n_kv_heads=2, window=64, seq_lens=(64,)),                      # n == w
+    dict(n_q_heads=8, n_kv_heads=2, window=64, seq_lens=(65, 200)),                  # one candidate
+])
+def test_split_query_groups(kw):
+    budget = min(max(kw["window"], 96), min(kw["seq_lens"]))   # between the window and the shortest n
+    cfg = get_config("llama8b_8k").scaled(n_layers=2, budget_per_head=budget, **kw)
+    compare_eviction(cfg)
+
