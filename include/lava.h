@@ -254,6 +254,14 @@ LAVA_API lava_status lava_evict_model_host(const lava_layer_desc* desc, int32_t 
 /* Number of kernel launches this library has enqueued from the calling process so far. */
 LAVA_API int64_t lava_launch_count(void);
 
+/* Which kernels lava_score_layer(s) will use for this geometry (host-side decision, no device
+ * work; honours LAVA_FORCE_GENERIC=1): 0 = CUDA-core path (fp32 inputs, head_dim 64, other
+ * windows), 1 = tensor-core path with one 128-row unit per KV head (Definition 1 with the GQA
+ * group maximum of Sec. 4.3 taken inside the kernel), 2 = tensor-core path with the query group
+ * of a KV head split into two units of at most 128 window-query rows whose maxima are merged
+ * in memory.  Returns -1 and sets lava_last_error() for an invalid descriptor. */
+LAVA_API int32_t lava_score_path(const lava_layer_desc* desc);
+
 #ifdef __cplusplus
 }
 #endif

@@ -77,6 +77,8 @@ def load_library():
     lib.lava_evict_model_host.restype = i32
     lib.lava_launch_count.restype = i64
     lib.lava_launch_count.argtypes = []
+    lib.lava_score_path.restype = i32
+    lib.lava_score_path.argtypes = [dp]
     for name in ("lava_poll_status", "lava_wo_norm", "lava_score_layer", "lava_score_layers",
                  "lava_layer_budgets", "lava_select_topk", "lava_select_topk_layers",
                  "lava_compact_kv", "lava_compact_kv_layers"):
@@ -335,6 +337,15 @@ def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC
 # ----------------------------------------------------------------------------- host buffers
 def lava_launch_count() -> int:
     return int(load_library().lava_launch_count())
+
+
+def lava_score_path(desc: LayerDesc) -> int:
+    """0 = CUDA-core path, 1 = tensor-core path, 2 = tensor-core path with split query groups."""
+    c = desc.to_c()
+    r = int(load_library().lava_score_path(ctypes.byref(c)))
+    if r < 0:
+        raise LavaError(1, load_library().lava_last_error().decode("utf-8", "replace"))
+    return r
 
 
 def lava_host_arena_bytes(desc: LayerDesc, n_layers: int, total_budget_rows: int) -> int:

@@ -134,6 +134,14 @@ int32_t lava_version(void) { return 100; }
 
 int64_t lava_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+int32_t lava_score_path(const lava_layer_desc* desc) {
+  Geom g;
+  if (make_geom(desc, &g) != LAVA_OK) return -1;
+  const char* force = getenv("LAVA_FORCE_GENERIC");
+  if (!sm100_supported(g) || (force && force[0] == '1')) return 0;
+  return g.group * g.window > 128 ? 2 : 1;
+}
+
 const char* lava_last_error(void) { return g_error; }
 
 size_t lava_workspace_bytes(const lava_layer_desc* desc, int32_t n_layers) {

@@ -86,3 +86,47 @@ def test_workspace_grows_with_layers_and_context():
     c = lava.lava_workspace_bytes(_desc(total_tokens=4096, k_stride_head=4096 * 64,
                                         v_stride_head=4096 * 64), 1)
     assert a < b and a < c
+
+
+def _config_desc(name):
+    from lava_workloads import get_config
+    cfg = get_config(name)
+    n, d = cfg.total_tokens, cfg.head_dim
+    return cfg, lava.LayerDesc(
+        n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads, head_dim=d, window=cfg.window,
+        pool_kind=cfg.pool_kind, pool_kernel=cfg.pool_kernel,
+        dtype=lava.LAVA_BF16 if cfg.dtype == "bf16" else lava.LAVA_F32, batch=cfg.batch,
+        max_seqlen=max(cfg.seq_lens), cu_seqlens=None, total_tokens=n, k_stride_head=n * d,
+        k_stride_tok=d, v_stride_head=n * d, v_stride_tok=d)
+
+
+@pytest.mark.parametrize("name,path", [
+    ("tiny", 0), ("llama8b_8k", 1), ("llama8b_32k", 1), ("gqa7_128k", 2)])
+def test_which_kernels_score_each_workload(name, path):
+    _, desc = _config_desc(name)
+    assert lava.lava_score_path(desc) == path
+
+
+def test_score_path_of_split_groups_and_of_what_stays_on_cuda_cores(monkeypatch):
+    base = dict(head_dim=128, dtype=lava.LAVA_BF16, total_tokens=4096, k_stride_head=4096 * 128,
+                k_stride_tok=128, v_stride_head=4096 * 128, v_stride_tok=128)
+    mk = lambda **kw: lava.LayerDesc(**{**base, **kw})
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=64)) == 2      # G 4 x w 64
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=64,
+                                   pool_kind=lava.LAVA_POOL_AVG, pool_kernel=5)) == 2
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=2, window=16)) == 2      # 8 heads per unit
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=128)) == 0     # 512 rows
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=48)) == 0      # odd window
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=2, window=16,
+                                   pool_kind=lava.LAVA_POOL_AVG, pool_kernel=5)) == 0  # avg: > 4 heads
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=32, dtype=lava.LAVA_F32)) == 0
+    monkeypatch.setenv("LAVA_FORCE_GENERIC", "1")
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=32)) == 0
+    with pytest.raises(lava.LavaError):
+        lava.lava_score_path(mk(n_q_heads=5, n_kv_heads=2, window=32))
+
+
+def test_workspace_for_a_model_also_serves_single_layers():
+    _, desc = _config_desc("llama8b_32k")
+    assert lava.lava_workspace_bytes(desc, 32) >= lava.lava_workspace_bytes(desc, 1)
+    assert lava.lava_workspace_bytes(desc, 32) >= lava.lava_workspace_bytes(desc, 7)

@@ -225,5 +225,13 @@ def test_host_buffer_path_equals_device_path():
 def test_split_query_groups(kw):
     budget = min(max(kw["window"], 96), min(kw["seq_lens"]))   # between the window and the shortest n
     cfg = get_config("llama8b_8k").scaled(n_layers=2, budget_per_head=budget, **kw)
+    n, d = cfg.total_tokens, cfg.head_dim
+    desc = lava.LayerDesc(n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads, head_dim=d,
+                          window=cfg.window, pool_kind=cfg.pool_kind, pool_kernel=cfg.pool_kernel,
+                          batch=cfg.batch, max_seqlen=max(cfg.seq_lens),
+                          cu_seqlens=torch.zeros(cfg.batch + 1, dtype=torch.int32) if cfg.batch > 1 else None,
+                          total_tokens=n, k_stride_head=n * d, k_stride_tok=d, v_stride_head=n * d,
+                          v_stride_tok=d)
+    assert lava.lava_score_path(desc) == 2, "this geometry must run as two units per KV head"
     compare_eviction(cfg)
 
