@@ -1,29 +1,31 @@
-// LAVa score, Blackwell path: bf16, head_dim 128, G*w <= 128, w in {16, 32, 64, 128}.
+// LAVa score, Blackwell path: bf16, head_dim 128, w in {16, 32, 64, 128}, up to 256 window-query
+// rows per KV head (a unit holds at most 128; larger query groups run as two units).
 //
 // One persistent, warp-specialised kernel (one CTA per SM, cooperative launch so that every CTA
 // is resident) runs two pipelines over 128-key tiles of K, both fed by TMA into 128B-swizzled
 // shared memory and contracted with tcgen05.mma into TMEM:
 //
-//   pass 1 (statistics)  S = Q_g K^T  (rows = the group's G*w window queries, columns = keys)
+//   pass 1 (statistics)  S = Q_g K^T  (rows = the unit's window queries, columns = keys)
 //       one thread per row reads its TMEM lane and keeps a running (max, sum of exp2) over the
 //       keys the query may see (Sec. 2: softmax over i <= j).  Work is dealt to CTAs in chunks
-//       of a few consecutive tiles of one head; a chunk's statistics leave the CTA once, through
-//       a publisher warp that also counts the head's published chunks.  Seven
-//       more warps stream the chunk's V rows for the value norm (Theorem 1: max_k ||V[k]||_1).
+//       of consecutive tiles of one head; a chunk's statistics leave the CTA once, through a
+//       publisher warp that also counts the head's published chunks.  Seven more warps stream
+//       the chunk's V rows for the value norm (Theorem 1: max_k ||V[k]||_1).
 //   pass 2 (scores)      S^T = K Q_g^T (rows = keys, columns = window queries)
 //       one thread per key: a_h[i] = (1/w) sum_t exp2(z - lse_t) per query head in registers,
 //       pooled over the token axis through shared memory, scaled by Vbar * c_hat, reduced with
 //       the GQA group maximum, written once; entropy sums go to ordered per-chunk slots
 //       (Definition 1, Sec. 4.2, Sec. 4.3, Sec. 5.1 pooling).
 //
-// The exponential unit bounds the kernel, so the eight consumer warps are not split by pass:
-// two groups of four warps each own one TMEM buffer of BOTH pipelines and take whichever of
-// their tiles is ready, which keeps two exp-issuing warps on every scheduler.
+// The exponentials bound the kernel, so the eight consumer warps are not split by pass: two
+// groups of four warps each own one TMEM buffer of BOTH pipelines and take their tiles in a
+// static order that alternates the passes, which keeps two exp-issuing warps on every scheduler.
 //
-// K is read from HBM once: pass 2 trails pass 1 by a bounded number of keys, so its tiles are
-// still in L2 (K tiles are loaded with an evict-last hint in pass 1 and evict-first in pass 2,
-// V rows with evict-first).  Every wait (mbarrier, head counters) is bounded in time; on
-// expiry the kernel sets LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
+// Pass 2 trails pass 1 by a bounded number of tiles (K tiles are loaded with an evict-last hint
+// in pass 1 and evict-first in pass 2, V rows with evict-first), so part of its K tiles are
+// still in L2; how many depends on the chunk length (see chunk_tiles_for).  Every wait
+// (mbarrier, head counters) is bounded in time; on expiry the kernel sets
+// LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
 #include <cuda.h>
 #include <stdlib.h>
 
