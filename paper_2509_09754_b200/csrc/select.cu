@@ -219,7 +219,8 @@ struct RegShared {
 
 template <int E>
 struct RegCfg {
-  static constexpr int kRep = E >= 32 ? 16 : 4;  // histogram copies
+  static constexpr int kRep = E >= 64 ? 16 : E >= 32 ? 8 : 4;  // histogram copies
+  static constexpr int kMinCtas = E >= 64 ? 1 : 2;  // CTAs per SM the kernel is compiled for
   static constexpr int kPad = E + 4;             // staging words per thread (bank spread)
   static constexpr int kStageWords = kThreads * kPad;
   static constexpr int kHistWords = kBins * kRep;
@@ -227,7 +228,7 @@ struct RegCfg {
 };
 
 template <int E>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, RegCfg<E>::kMinCtas)
 select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budget, int* keep_idx,
                        int* head_offsets) {
   using Cfg = RegCfg<E>;
