@@ -251,11 +251,32 @@ LAVA_API lava_status lava_evict_model_host(const lava_layer_desc* desc, int32_t 
                                            int32_t* head_offsets, void* k_out, void* v_out,
                                            void* arena, size_t arena_bytes, void* stream);
 
+/* Tuning and test knobs (no counterpart in the paper).  Process-wide; the defaults come from the
+ * environment variables named below, read once when the library first needs an option, so no
+ * call on the hot path reads the environment.  Set them while no call of this library is running.
+ *   "select_cluster"     0 = choose by size (default), 8 or 16 CTAs per selection cluster
+ *                        (LAVA_SELECT_CLUSTER)
+ *   "score_kernel"       0 = choose by geometry (default), 1 = two-pass tensor-core kernel,
+ *                        2 = single-pass kernel that keeps the logits in tensor memory where the
+ *                        geometry allows it (LAVA_SCORE_KERNEL)
+ *   "score_chunk_tiles"  0 = choose per launch, else 1..64 key tiles per chunk of the two-pass
+ *                        kernel (LAVA_SM100_CHUNK_TILES)
+ *   "score_lead_tiles"   -1 = choose, else extra tiles pass 1 leads pass 2 by (LAVA_SM100_LEAD_TILES)
+ *   "force_generic"      1 = score on the CUDA-core path whatever the geometry (LAVA_FORCE_GENERIC)
+ *   "wait_limit_cycles"  SM cycles after which a device-side wait on another warp role or CTA
+ *                        gives up and sets LAVA_DEV_WAIT_EXPIRED (default 2^32, about two seconds;
+ *                        LAVA_WAIT_LIMIT_CYCLES).  Waits for copies already in flight keep the
+ *                        default so that a kernel never exits under a running copy.
+ * lava_set_option returns LAVA_ERR_INVALID_ARG for an unknown name or a value out of range;
+ * lava_get_option returns INT64_MIN for an unknown name. */
+LAVA_API lava_status lava_set_option(const char* name, int64_t value);
+LAVA_API int64_t lava_get_option(const char* name);
+
 /* Number of kernel launches this library has enqueued from the calling process so far. */
 LAVA_API int64_t lava_launch_count(void);
 
 /* Which kernels lava_score_layer(s) will use for this geometry (host-side decision, no device
- * work; honours LAVA_FORCE_GENERIC=1): 0 = CUDA-core path (fp32 inputs, head_dim 64, other
+ * work; honours the "force_generic" option): 0 = CUDA-core path (fp32 inputs, head_dim 64, other
  * windows), 1 = tensor-core path with one 128-row unit per KV head (Definition 1 with the GQA
  * group maximum of Sec. 4.3 taken inside the kernel), 2 = tensor-core path with the query group
  * of a KV head split into two units of at most 128 window-query rows whose maxima are merged

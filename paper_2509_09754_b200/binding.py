@@ -79,6 +79,10 @@ def load_library():
     lib.lava_launch_count.argtypes = []
     lib.lava_score_path.restype = i32
     lib.lava_score_path.argtypes = [dp]
+    lib.lava_set_option.restype = i32
+    lib.lava_set_option.argtypes = [ctypes.c_char_p, i64]
+    lib.lava_get_option.restype = i64
+    lib.lava_get_option.argtypes = [ctypes.c_char_p]
     for name in ("lava_poll_status", "lava_wo_norm", "lava_score_layer", "lava_score_layers",
                  "lava_layer_budgets", "lava_select_topk", "lava_select_topk_layers",
                  "lava_compact_kv", "lava_compact_kv_layers"):
@@ -335,6 +339,18 @@ def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC
 
 
 # ----------------------------------------------------------------------------- host buffers
+def lava_set_option(name: str, value: int) -> None:
+    """Process-wide tuning / test knob (see lava.h for the names)."""
+    _check(load_library().lava_set_option(name.encode(), int(value)))
+
+
+def lava_get_option(name: str) -> int:
+    v = int(load_library().lava_get_option(name.encode()))
+    if v == -(1 << 63):
+        raise LavaError(1, lava_last_error())
+    return v
+
+
 def lava_launch_count() -> int:
     return int(load_library().lava_launch_count())
 

@@ -52,7 +52,8 @@ lava_status launch_compact(const Geom& g, int n_layers, const void* k, const voi
   // Row counts live on the device, so the grid is sized for the bandwidth, not the data: enough
   // blocks per (layer, sequence, head) to fill the GPU, each striding over the head's rows.
   const int heads_total = n_layers * g.batch * g.n_kv_heads;
-  int blocks_per_head = (148 * 8 + heads_total - 1) / heads_total;
+  const int sms = sm_count() > 0 ? sm_count() : 1;
+  int blocks_per_head = (sms * 8 + heads_total - 1) / heads_total;
   if (blocks_per_head < 1) blocks_per_head = 1;
   const int max_useful = (g.max_seqlen + 15) / 16;
   if (blocks_per_head > max_useful) blocks_per_head = max_useful;

@@ -2,6 +2,7 @@
 // stream while earlier layers are scored, then runs budgets, selection and compaction and
 // copies the results back.  Only copies and calls into the device-pointer entry points happen
 // here; all arithmetic stays in the kernels.
+#include <mutex>
 #include <vector>
 
 #include "lava_internal.cuh"
@@ -16,6 +17,13 @@ struct HostPathState {
 };
 
 HostPathState g_state[64];
+std::mutex g_state_mutex;  // guards the creation of a device's stream and events
+
+// The host arrays are dense whatever strides the caller's descriptor carries.
+void set_dense_layout(lava_layer_desc* d) {
+  d->k_stride_tok = d->v_stride_tok = d->head_dim;
+  d->k_stride_head = d->v_stride_head = d->total_tokens * d->head_dim;
+}
 
 size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
@@ -70,8 +78,10 @@ size_t lava_host_arena_bytes(const lava_layer_desc* desc, int32_t n_layers,
                              int64_t total_budget_rows) {
   Geom g;
   if (n_layers < 1 || total_budget_rows < 0) return 0;
+  if (!desc) return 0;
   lava_layer_desc d = *desc;
   d.cu_seqlens = d.batch > 1 ? reinterpret_cast<const int32_t*>(16) : nullptr;
+  set_dense_layout(&d);
   if (make_geom(&d, &g) != LAVA_OK) return 0;
   return arena_layout(&d, n_layers, total_budget_rows).total;
 }
@@ -113,11 +123,10 @@ lava_status lava_evict_model_host(const lava_layer_desc* desc, int32_t n_layers,
     return fail(LAVA_ERR_INVALID_ARG, "seq_lens do not sum to total_tokens");
 
   lava_layer_desc d = *desc;
+  set_dense_layout(&d);
+  d.max_seqlen = max_len;
   const Arena a = arena_layout(&d, n_layers, rows);
   d.cu_seqlens = d.batch > 1 ? reinterpret_cast<const int32_t*>(base + a.cu) : nullptr;
-  d.max_seqlen = max_len;
-  d.k_stride_tok = d.v_stride_tok = d.head_dim;
-  d.k_stride_head = d.v_stride_head = d.total_tokens * d.head_dim;
   Geom g;
   lava_status rc = make_geom(&d, &g);
   if (rc != LAVA_OK) return rc;
@@ -129,17 +138,20 @@ lava_status lava_evict_model_host(const lava_layer_desc* desc, int32_t n_layers,
   if (rc != LAVA_OK) return rc;
   if (dev < 0 || dev >= 64) return fail(LAVA_ERR_UNSUPPORTED, "device index out of range");
   HostPathState& st = g_state[dev];
-  if (!st.copy_stream) {
-    rc = check_cuda(cudaStreamCreateWithFlags(&st.copy_stream, cudaStreamNonBlocking), "stream create");
-    if (rc != LAVA_OK) return rc;
-    rc = check_cuda(cudaEventCreateWithFlags(&st.start, cudaEventDisableTiming), "event create");
-    if (rc != LAVA_OK) return rc;
-  }
-  while ((int)st.layer_ready.size() < n_layers) {
-    cudaEvent_t e;
-    rc = check_cuda(cudaEventCreateWithFlags(&e, cudaEventDisableTiming), "event create");
-    if (rc != LAVA_OK) return rc;
-    st.layer_ready.push_back(e);
+  {
+    std::lock_guard<std::mutex> lock(g_state_mutex);
+    if (!st.copy_stream) {
+      rc = check_cuda(cudaStreamCreateWithFlags(&st.copy_stream, cudaStreamNonBlocking), "stream create");
+      if (rc != LAVA_OK) return rc;
+      rc = check_cuda(cudaEventCreateWithFlags(&st.start, cudaEventDisableTiming), "event create");
+      if (rc != LAVA_OK) return rc;
+    }
+    while ((int)st.layer_ready.size() < n_layers) {
+      cudaEvent_t e;
+      rc = check_cuda(cudaEventCreateWithFlags(&e, cudaEventDisableTiming), "event create");
+      if (rc != LAVA_OK) return rc;
+      st.layer_ready.push_back(e);
+    }
   }
 
   cudaStream_t main_s = (cudaStream_t)stream, copy_s = st.copy_stream;

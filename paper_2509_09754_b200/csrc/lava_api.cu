@@ -29,6 +29,39 @@ lava_status check_cuda(cudaError_t e, const char* what) {
   return fail(LAVA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+static long long env_ll(const char* name, long long lo, long long hi, long long dflt) {
+  const char* e = getenv(name);
+  if (!e || !*e) return dflt;
+  const long long v = atoll(e);
+  return (v < lo || v > hi) ? dflt : v;
+}
+
+Options& options() {
+  static Options opt = [] {
+    Options o;
+    o.select_cluster = (int)env_ll("LAVA_SELECT_CLUSTER", 8, 16, 0);
+    if (o.select_cluster != 8 && o.select_cluster != 16) o.select_cluster = 0;
+    o.score_chunk_tiles = (int)env_ll("LAVA_SM100_CHUNK_TILES", 1, 64, 0);
+    o.score_lead_tiles = (int)env_ll("LAVA_SM100_LEAD_TILES", 0, 4096, -1);
+    o.force_generic = (int)env_ll("LAVA_FORCE_GENERIC", 0, 1, 0);
+    o.score_kernel = (int)env_ll("LAVA_SCORE_KERNEL", 0, 2, 0);
+    o.wait_limit_cycles = env_ll("LAVA_WAIT_LIMIT_CYCLES", 1, 1ll << 40, 1ll << 32);
+    return o;
+  }();
+  return opt;
+}
+
+int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -137,12 +170,45 @@ int64_t lava_launch_count(void) { return g_launches.load(std::memory_order_relax
 int32_t lava_score_path(const lava_layer_desc* desc) {
   Geom g;
   if (make_geom(desc, &g) != LAVA_OK) return -1;
-  const char* force = getenv("LAVA_FORCE_GENERIC");
-  if (!sm100_supported(g) || (force && force[0] == '1')) return 0;
+  if (!sm100_supported(g) || options().force_generic) return 0;
   return g.group * g.window > 128 ? 2 : 1;
 }
 
 const char* lava_last_error(void) { return g_error; }
+
+static long long* option_slot(const char* name, long long* lo, long long* hi, int** as_int) {
+  Options& o = options();
+  *as_int = nullptr;
+  if (!name) return nullptr;
+  if (!strcmp(name, "select_cluster")) { *lo = 0; *hi = 16; *as_int = &o.select_cluster; }
+  else if (!strcmp(name, "score_chunk_tiles")) { *lo = 0; *hi = 64; *as_int = &o.score_chunk_tiles; }
+  else if (!strcmp(name, "score_lead_tiles")) { *lo = -1; *hi = 4096; *as_int = &o.score_lead_tiles; }
+  else if (!strcmp(name, "force_generic")) { *lo = 0; *hi = 1; *as_int = &o.force_generic; }
+  else if (!strcmp(name, "score_kernel")) { *lo = 0; *hi = 2; *as_int = &o.score_kernel; }
+  else if (!strcmp(name, "wait_limit_cycles")) { *lo = 1; *hi = 1ll << 40; return &o.wait_limit_cycles; }
+  return nullptr;
+}
+
+lava_status lava_set_option(const char* name, int64_t value) {
+  long long lo = 0, hi = 0;
+  int* as_int = nullptr;
+  long long* slot = option_slot(name, &lo, &hi, &as_int);
+  if (!slot && !as_int) return fail(LAVA_ERR_INVALID_ARG, "unknown option '%s'", name ? name : "(null)");
+  if (value < lo || value > hi || (as_int == &options().select_cluster && value != 0 && value != 8 && value != 16))
+    return fail(LAVA_ERR_INVALID_ARG, "option %s: value %lld out of range", name, (long long)value);
+  if (as_int) *as_int = (int)value; else *slot = value;
+  return LAVA_OK;
+}
+
+int64_t lava_get_option(const char* name) {
+  long long lo = 0, hi = 0;
+  int* as_int = nullptr;
+  long long* slot = option_slot(name, &lo, &hi, &as_int);
+  if (as_int) return *as_int;
+  if (slot) return *slot;
+  fail(LAVA_ERR_INVALID_ARG, "unknown option '%s'", name ? name : "(null)");
+  return INT64_MIN;
+}
 
 size_t lava_workspace_bytes(const lava_layer_desc* desc, int32_t n_layers) {
   Geom g;
@@ -198,8 +264,7 @@ lava_status lava_score_layers(const lava_layer_desc* desc, int32_t n_layers, con
     return fail(LAVA_ERR_WORKSPACE, "workspace too small: %zu < %zu bytes", workspace_bytes,
                 lay.total);
   if (!aligned16(workspace)) return fail(LAVA_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
-  const char* force = getenv("LAVA_FORCE_GENERIC");
-  if (sm100_supported(g) && !(force && force[0] == '1'))
+  if (sm100_supported(g) && !options().force_generic)
     return launch_score_sm100(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
                               v_layer_stride, vbar_in, scores, vbar_out, entropy,
                               (char*)workspace, lay.off_sm100, (cudaStream_t)stream);

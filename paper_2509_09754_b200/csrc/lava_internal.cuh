@@ -53,6 +53,19 @@ struct Workspace {
 };
 Workspace workspace_layout(const lava_layer_desc* d, int n_layers);
 
+// Tuning and test knobs of the library (lava_set_option / lava_get_option).  The defaults come from
+// the environment, read once when the first option is looked at; nothing on a call path calls getenv.
+struct Options {
+  int select_cluster;      // 0: choose by size, else 8 or 16 CTAs per selection cluster
+  int score_chunk_tiles;   // 0: choose per launch, else tiles per chunk of the two-pass score kernel
+  int score_lead_tiles;    // -1: choose, else the extra tiles pass 1 leads pass 2 by
+  int force_generic;       // 1: score on the CUDA-core path whatever the geometry
+  int score_kernel;        // 0: choose, 1: two-pass kernel, 2: single-pass (logits kept in TMEM)
+  long long wait_limit_cycles;  // SM cycles after which a device-side wait that may be abandoned gives up
+};
+Options& options();
+int sm_count();            // multiprocessors of the current device (cached per device), 0 on error
+
 // Host-side error plumbing.
 lava_status fail(lava_status st, const char* fmt, ...);
 lava_status check_cuda(cudaError_t e, const char* what);

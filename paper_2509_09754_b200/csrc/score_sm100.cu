@@ -27,7 +27,6 @@
 // (mbarrier, head counters) is bounded in time; on expiry the kernel sets
 // LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "lava_internal.cuh"
 
@@ -43,7 +42,7 @@ constexpr int kStages = 2;           // K stages per pipeline
 constexpr int kMaxBatch = 512;       // sequences the in-kernel chunk schedule can index
 constexpr uint32_t kTileBytes = 128 * 128 * 2;  // one [128 x 128] bf16 tile = 2 swizzled blocks
 constexpr uint32_t kHalfBytes = kTileBytes / 2;
-constexpr long long kWaitCycles = 1ll << 32;  // every wait gives up after about two seconds
+constexpr long long kWaitCycles = 1ll << 32;  // the drain waits at exit give up after about two seconds
 
 // shared memory map (bytes from a 1024-aligned base)
 // Two small operands in the un-swizzled K-major layout (8 x 16-byte core matrices, 128 B apart
@@ -76,6 +75,7 @@ struct Misc {
   unsigned long long drain, drain2;
   uint32_t tmem_base;
   volatile int abort_flag;
+  long long wait_cycles;              // limit of the waits that an abort may end (launch parameter)
   int sched_total1, sched_total2;     // chunks per layer of pass 1 / pass 2
   int lead_tiles;                     // tile slots pass 1 runs ahead of pass 2 in a CTA's order
   alignas(16) float pub[2][2][128];   // [slot][group][query]: log2-sum-exp of a finished chunk
@@ -94,6 +94,7 @@ struct Sm100Params {
   int lead_extra;           // tiles pass 1 leads pass 2 by, beyond what head completion needs
   int split;                // 1: every KV head is scored as two halves of its query group
   int g0;                   // query heads in the first half (split mode)
+  long long wait_cycles;    // SM cycles after which a wait on another role or CTA gives up
   const float* vbar_in;
   float* scores;
   float* vbar_out;
@@ -327,7 +328,7 @@ __device__ inline bool wait_bar(uint32_t bar, uint32_t parity, Misc* m, unsigned
   for (;;) {
     if (mbar_try(bar, parity, 1000)) return true;
     if (heed_abort && m->abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) break;
+    if (clock64() - t0 > (heed_abort ? m->wait_cycles : kWaitCycles)) break;
   }
   give_up(m, status);
   return false;
@@ -404,6 +405,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     int c1 = 0, c2 = 0;
     if ((int)threadIdx.x < g.batch) {
       const SeqInfo s = seq_info(g, threadIdx.x);
+      if (s.n < g.window && blockIdx.x == 0) atomicOr(p.status, LAVA_DEV_SHORT_SEQUENCE);
       c1 = ceil_div(ceil_div(s.n, kTile), p.chunk_tiles);
       c2 = ceil_div(ceil_div(s.prefix, p.out_keys), p.chunk_tiles);
     }
@@ -480,6 +482,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     mbar_init(smem_u32(&m->drain), 1);
     mbar_init(smem_u32(&m->drain2), 1);
     m->abort_flag = 0;
+    m->wait_cycles = p.wait_cycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -555,7 +558,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
                (want_v && ld_acquire(&p.vcount[ck.rhead]) < want_v)) {
           if (m->abort_flag) break;
           __nanosleep(100);
-          if (clock64() - t0 > kWaitCycles) give_up(m, p.status);
+          if (clock64() - t0 > m->wait_cycles) give_up(m, p.status);
         }
         ok = !m->abort_flag &&
              wait_bar(smem_u32(&m->prep_empty[slot]), (uint32_t)((j >> 1) & 1) ^ 1, m, p.status);
@@ -1265,7 +1268,7 @@ size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 // of statistics, so chunks should be long; but the launch needs many more chunks than CTAs to
 // balance (chunks are dealt round-robin), and a head finishes pass 1 sooner when more CTAs
 // share it.  Default: about twelve chunks per CTA, between 4 and 32 tiles.  LAVA_SM100_CHUNK_TILES
-// overrides it.
+// overrides it (option "score_chunk_tiles").
 constexpr int kMinChunkTiles = 4, kMaxChunkTiles = 32;
 
 // Query groups of more than 128 window-query rows are scored as two halves (each a unit of its
@@ -1275,16 +1278,11 @@ int sm100_first_half(const Geom& g) {
   return g.group * g.window > 128 ? (g.group + 1) / 2 : 0;
 }
 int chunk_tiles_for(const Geom& g, int n_layers) {
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = getenv("LAVA_SM100_CHUNK_TILES");
-    const int v = e ? atoi(e) : 0;
-    forced = (v >= 1 && v <= 64) ? v : 0;
-  }
-  if (forced) return forced;
+  if (options().score_chunk_tiles > 0) return options().score_chunk_tiles;
   const long long tiles = (long long)n_layers * (g.n_kv_heads << (sm100_first_half(g) ? 1 : 0)) *
                           ceil_div((int)g.total_tokens, kTile);
-  const long long r = tiles / (148 * 12);
+  const int sms = sm_count() > 0 ? sm_count() : 148;  // without a device: the part this is tuned for
+  const long long r = tiles / ((long long)sms * 12);
   return (int)(r < kMinChunkTiles ? kMinChunkTiles : r > kMaxChunkTiles ? kMaxChunkTiles : r);
 }
 
@@ -1292,12 +1290,7 @@ int chunk_tiles_for(const Geom& g, int n_layers) {
 // statistics take to be published and folded, and the skew between CTAs): half a chunk.
 // LAVA_SM100_LEAD_TILES overrides it.
 int lead_extra_for(int chunk_tiles) {
-  static int forced = -2;
-  if (forced == -2) {
-    const char* e = getenv("LAVA_SM100_LEAD_TILES");
-    const int v = e ? atoi(e) : -1;
-    forced = (v >= 0 && v <= 4096) ? v : -1;
-  }
+  const int forced = options().score_lead_tiles;
   return forced >= 0 ? forced : (chunk_tiles + 1) / 2;
 }
 
@@ -1381,11 +1374,9 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
       return fail(LAVA_ERR_CUDA, "tensor map for K could not be encoded");
   }
 
-  int dev = 0, sms = 0;
-  lava_status rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
-  if (rc != LAVA_OK) return rc;
-  rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "SM count");
-  if (rc != LAVA_OK) return rc;
+  const int sms = sm_count();
+  if (sms <= 0) return fail(LAVA_ERR_CUDA, "the multiprocessor count of the device is not available");
+  lava_status rc = LAVA_OK;
 
   Sm100Params p;
   p.g = g;
@@ -1397,6 +1388,7 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
   p.lead_extra = lead_extra_for(lay.chunk_tiles);
   p.g0 = sm100_first_half(g);
   p.split = p.g0 ? 1 : 0;
+  p.wait_cycles = options().wait_limit_cycles;
   p.vbar_in = vbar_in;
   p.scores = scores;
   p.vbar_out = vbar_out;

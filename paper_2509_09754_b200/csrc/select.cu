@@ -10,7 +10,6 @@
 // contiguous eighth of the flat array.  Histograms and counts are exchanged through
 // distributed shared memory with hardware cluster barriers (no spin waits, no global atomics).
 #include <cooperative_groups.h>
-#include <stdlib.h>
 
 #include "lava_internal.cuh"
 
@@ -461,9 +460,9 @@ lava_status launch_select(const Geom& g, int n_layers, const float* scores,
   const int problems = n_layers * g.batch;
   // 16 CTAs once a cluster of 8 would need 64 keys per thread: at 32 keys per thread two CTAs
   // share an SM
-  const char* cs_env = getenv("LAVA_SELECT_CLUSTER");
   int csize = m_max <= 8LL * (kRegMaxPerCta / 2) ? 8 : 16;
-  if (cs_env && atoi(cs_env) == 8 && m_max <= 8LL * kRegMaxPerCta) csize = 8;
+  if (options().select_cluster == 8 && m_max <= 8LL * kRegMaxPerCta) csize = 8;
+  if (options().select_cluster == 16) csize = 16;
   if (m_max <= (long long)csize * kRegMaxPerCta) {
     const long long per = (m_max + csize - 1) / csize;
     const int e = (int)((per + kThreads - 1) / kThreads);  // keys per thread

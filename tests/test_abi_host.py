@@ -120,8 +120,12 @@ def test_score_path_of_split_groups_and_of_what_stays_on_cuda_cores(monkeypatch)
     assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=2, window=16,
                                    pool_kind=lava.LAVA_POOL_AVG, pool_kernel=5)) == 0  # avg: > 4 heads
     assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=32, dtype=lava.LAVA_F32)) == 0
-    monkeypatch.setenv("LAVA_FORCE_GENERIC", "1")
-    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=32)) == 0
+    lava.lava_set_option("force_generic", 1)
+    try:
+        assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=32)) == 0
+    finally:
+        lava.lava_set_option("force_generic", 0)
+    assert lava.lava_score_path(mk(n_q_heads=32, n_kv_heads=8, window=32)) == 1
     with pytest.raises(lava.LavaError):
         lava.lava_score_path(mk(n_q_heads=5, n_kv_heads=2, window=32))
 
@@ -130,3 +134,34 @@ def test_workspace_for_a_model_also_serves_single_layers():
     _, desc = _config_desc("llama8b_32k")
     assert lava.lava_workspace_bytes(desc, 32) >= lava.lava_workspace_bytes(desc, 1)
     assert lava.lava_workspace_bytes(desc, 32) >= lava.lava_workspace_bytes(desc, 7)
+
+
+def test_options_round_trip_and_reject_bad_values():
+    for name, value in (("select_cluster", 16), ("score_chunk_tiles", 8), ("score_lead_tiles", 5),
+                        ("wait_limit_cycles", 12345), ("score_kernel", 1)):
+        before = lava.lava_get_option(name)
+        lava.lava_set_option(name, value)
+        assert lava.lava_get_option(name) == value
+        lava.lava_set_option(name, before)
+        assert lava.lava_get_option(name) == before
+    lib = lava.load_library()
+    assert lib.lava_set_option(b"select_cluster", 12) == 1
+    assert lib.lava_set_option(b"wait_limit_cycles", 0) == 1
+    assert lib.lava_set_option(b"no_such_option", 1) == 1
+    assert lib.lava_set_option(None, 1) == 1
+    assert "unknown option" in lava.lava_last_error()
+    with pytest.raises(lava.LavaError):
+        lava.lava_get_option("no_such_option")
+
+
+def test_host_buffer_arena_size_ignores_the_descriptor_strides():
+    """The host arrays of lava_evict_model_host are dense, so whatever strides the descriptor
+    carries (zeros included) must give the same arena size."""
+    cfg, desc = _config_desc("llama8b_8k")
+    dense = lava.lava_host_arena_bytes(desc, 4, 4 * 8 * 512)
+    import dataclasses
+    zero = dataclasses.replace(desc, k_stride_head=0, k_stride_tok=0, v_stride_head=0, v_stride_tok=0)
+    odd = dataclasses.replace(desc, k_stride_tok=1024, v_stride_tok=256, k_stride_head=8)
+    assert dense > 0
+    assert lava.lava_host_arena_bytes(zero, 4, 4 * 8 * 512) == dense
+    assert lava.lava_host_arena_bytes(odd, 4, 4 * 8 * 512) == dense

@@ -318,6 +318,48 @@ def test_masked_attention_distance_identity():
         assert lhs == pytest.approx(2.0 * (a * (1 - m)).sum(), abs=1e-13)
 
 
+def test_layer_output_loss_closed_form_with_identity_values_and_projection():
+    """Lemma 1 with V_h = I (d_h = n) and W_O = I: the concatenated rows are A_h - A_hat_h, so
+    the loss is sum_h ||A_h - A_hat_h||_1 = 2 * (evicted attention mass over all heads), by the
+    identity in the proof of Theorem 1.  A version that drops a head or a term fails."""
+    rng = np.random.RandomState(31)
+    n_heads, n = 3, 7
+    att = rng.rand(n_heads, n)
+    att /= att.sum(axis=1, keepdims=True)
+    v = np.stack([np.eye(n)] * n_heads)
+    w_o = np.eye(n_heads * n)
+    for trial in range(20):
+        masks = (rng.rand(n_heads, n) < 0.6).astype(np.float64)
+        masks[:, -1] = 1.0                                   # something is always kept
+        want = 2.0 * float((att * (1.0 - masks)).sum())
+        assert O.layer_output_loss(att, v, w_o, masks) == pytest.approx(want, abs=1e-13)
+    # per-head contributions add up: with one head's mask full, that head contributes nothing
+    masks = np.ones((n_heads, n))
+    masks[1, :3] = 0.0
+    assert O.layer_output_loss(att, v, w_o, masks) == pytest.approx(2.0 * att[1, :3].sum(), abs=1e-13)
+
+
+def test_layer_output_loss_hand_worked_two_heads_with_projection():
+    """Lemma 1 by hand: 2 heads, n = 3, d_h = 2, a W_O that mixes and flips signs.
+
+    head 0: A = (.5, .3, .2), mask (1, 0, 1) -> A_hat = (5/7, 0, 2/7), A - A_hat = (-3/14, 3/10, -3/35)
+            V = [[1, 0], [0, 2], [1, 1]]     -> (A - A_hat) V = (-3/10, 18/35)
+    head 1: A = (.2, .2, .6), mask (0, 1, 1) -> A_hat = (0, 1/4, 3/4), A - A_hat = (1/5, -1/20, -3/20)
+            V = [[2, 1], [0, 1], [1, 0]]     -> (A - A_hat) V = (1/4, 3/20)
+    Cat = (-3/10, 18/35, 1/4, 3/20);  W_O = [[1, -1], [2, 0], [0, 3], [-1, 1]]
+    Cat W_O = (-3/10 + 36/35 - 3/20,  3/10 + 3/4 + 3/20) = (81/140, 6/5);  L1 norm = 249/140.
+    """
+    att = np.array([[0.5, 0.3, 0.2], [0.2, 0.2, 0.6]])
+    masks = np.array([[1.0, 0.0, 1.0], [0.0, 1.0, 1.0]])
+    v = np.array([[[1.0, 0.0], [0.0, 2.0], [1.0, 1.0]], [[2.0, 1.0], [0.0, 1.0], [1.0, 0.0]]])
+    w_o = np.array([[1.0, -1.0], [2.0, 0.0], [0.0, 3.0], [-1.0, 1.0]])
+    assert O.layer_output_loss(att, v, w_o, masks) == pytest.approx(249.0 / 140.0, abs=1e-14)
+    # the bound of Theorem 1 for the same case: C_hat = max row sum of |W_O| = 3,
+    # Vbar = (2, 3), evicted mass (.3, .2): 2 * 3 * (2 * .3 + 3 * .2) = 7.2
+    assert O.wo_norm(w_o) == 3.0
+    assert O.loss_upper_bound(att, v, w_o, masks) == pytest.approx(7.2, abs=1e-14)
+
+
 def test_bound_holds_and_topk_minimises_it_by_enumeration():
     """w = 1, MHA, no pooling: every subset obeys Theorem 1; top-k minimises the bound."""
     hq = hkv = 2
