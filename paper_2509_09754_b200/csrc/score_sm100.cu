@@ -26,12 +26,12 @@
 // still in L2; how many depends on the chunk length (see chunk_tiles_for).  Every wait
 // (mbarrier, head counters) is bounded in time; on expiry the kernel sets
 // LAVA_DEV_WAIT_EXPIRED, drains its copies, frees TMEM and returns.
-#include <cuda.h>
-
-#include "lava_internal.cuh"
+#include "sm100_ptx.cuh"
 
 namespace lava {
 namespace {
+
+using namespace sm100;
 
 constexpr int kTile = 128;           // keys per tile
 constexpr int kThreads = 640;        // 20 warps: 5 service, 8 consumer, 7 value-norm
@@ -42,7 +42,6 @@ constexpr int kStages = 2;           // K stages per pipeline
 constexpr int kMaxBatch = 512;       // sequences the in-kernel chunk schedule can index
 constexpr uint32_t kTileBytes = 128 * 128 * 2;  // one [128 x 128] bf16 tile = 2 swizzled blocks
 constexpr uint32_t kHalfBytes = kTileBytes / 2;
-constexpr long long kWaitCycles = 1ll << 32;  // the drain waits at exit give up after about two seconds
 
 // shared memory map (bytes from a 1024-aligned base)
 // Two small operands in the un-swizzled K-major layout (8 x 16-byte core matrices, 128 B apart
@@ -108,231 +107,6 @@ struct Sm100Params {
   float2* ent_part;         // [heads_total][cph2_max][8 consumer warps] (sum s, sum s ln s)
   unsigned* status;
 };
-
-// ------------------------------------------------------------------------------------------
-// PTX wrappers
-// ------------------------------------------------------------------------------------------
-__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ inline void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ inline void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ inline void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// Blocking form: the thread is suspended until the phase completes or a time limit (at most
-// about `ns` nanoseconds) passes, so a waiting warp does not occupy issue slots.
-__device__ inline bool mbar_try(uint32_t bar, uint32_t parity, uint32_t ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(ns)
-      : "memory");
-  return ok != 0;
-}
-__device__ inline uint64_t policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ inline uint64_t policy_evict_last() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ inline void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
-                                   uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-      : "memory");
-}
-__device__ inline void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
-                                   int c3, uint32_t bar, uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      ".L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
-      : "memory");
-}
-__device__ inline void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
-               "r"(ncols)
-               : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ inline void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
-               : "memory");
-}
-__device__ inline void tc_fence_before() {
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ inline void tc_fence_after() {
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ inline void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = N = 128, K = 16
-__device__ inline void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                 uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// 32 consecutive fp32 columns of this thread's TMEM lane: issue, and (separately) wait.  The
-// wait names the destination registers so that no use of them can be scheduled before it.
-__device__ inline void tmem_ld32_issue(uint32_t taddr, float* v) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
-        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ inline void tmem_ld_wait(float* v) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile(
-      "tcgen05.wait::ld.sync.aligned;"
-      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
-        "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]),
-        "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]),
-        "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
-        "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-      :
-      : "memory");
-}
-__device__ inline float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// Sum of 32 values by a fixed tree (i with i + 16, then + 8, + 4, then ((0 + 1) + (2 + 3))); the
-// wide levels use the packed two-lane fp32 add, which rounds each lane like the scalar add.
-__device__ inline float tree_sum32(float (&c)[32]) {
-#pragma unroll
-  for (int i = 0; i < 16; i += 2) {
-    const float2 r = __fadd2_rn(make_float2(c[i], c[i + 1]), make_float2(c[i + 16], c[i + 17]));
-    c[i] = r.x;
-    c[i + 1] = r.y;
-  }
-#pragma unroll
-  for (int i = 0; i < 8; i += 2) {
-    const float2 r = __fadd2_rn(make_float2(c[i], c[i + 1]), make_float2(c[i + 8], c[i + 9]));
-    c[i] = r.x;
-    c[i + 1] = r.y;
-  }
-#pragma unroll
-  for (int i = 0; i < 4; i += 2) {
-    const float2 r = __fadd2_rn(make_float2(c[i], c[i + 1]), make_float2(c[i + 4], c[i + 5]));
-    c[i] = r.x;
-    c[i + 1] = r.y;
-  }
-  return (c[0] + c[1]) + (c[2] + c[3]);
-}
-__device__ inline float fast_log2(float x) {
-  float y;
-  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// log2(2^a + 2^b) for values that may be -inf
-__device__ inline float lse2(float a, float b) {
-  const float hi = fmaxf(a, b), lo = fminf(a, b);
-  if (lo == -INFINITY) return hi;
-  return hi + fast_log2(1.0f + fast_exp2(lo - hi));
-}
-// counter increment that publishes this thread's earlier writes (and those ordered before it by
-// a barrier)
-__device__ inline void red_add_release(int* p, int v) {
-  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ inline int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-// 16 bytes of a value row, read once.  The plain streaming form: the variant with an L2 cache
-// hint operand and L1::no_allocate made the whole kernel a tenth slower.
-__device__ inline uint4 ld_stream16(const void* p) {
-  uint4 r;
-  asm volatile("ld.global.cs.v4.u32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p));
-  return r;
-}
-
-// D (+)= A * B on the register-operand tensor path: A 16 x 16 bf16 (row-major fragment a0..a3),
-// B 16 x 8 bf16 (b0, b1), D 16 x 8 fp32.  Thread (g = lane / 4, t = lane % 4) holds d0, d1 of
-// row g and d2, d3 of row g + 8; a0, a2 belong to row g and a1, a3 to row g + 8.
-__device__ inline void mma_bf16_16816(float& d0, float& d1, float& d2, float& d3, uint32_t a0,
-                                      uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                      uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
-      "{%8, %9}, {%0, %1, %2, %3};"
-      : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 B apart.
-__device__ inline uint64_t make_desc(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;            // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;  // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;            // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;            // 128-byte swizzle
-  return d;
-}
-// The same for an un-swizzled K-major operand of 16 columns: core matrices of 8 rows x 16 bytes,
-// 2048 B apart along k (leading offset) and 128 B apart along the rows (stride offset).
-__device__ inline uint64_t make_desc_plain(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)(2048 >> 4) << 16;
-  d |= (uint64_t)(128 >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  return d;
-}
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-
-__device__ inline void give_up(Misc* m, unsigned* status) {
-  m->abort_flag = 1;
-  atomicOr(status, LAVA_DEV_WAIT_EXPIRED);
-}
-
-// Bounded mbarrier wait.  Returns false once the CTA is aborting (unless heed_abort is false:
-// the drain waits at exit must outlast an abort to let copies in flight land).
-__device__ inline bool wait_bar(uint32_t bar, uint32_t parity, Misc* m, unsigned* status,
-                                bool heed_abort = true) {
-  if (mbar_try(bar, parity, 1000)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    if (mbar_try(bar, parity, 1000)) return true;
-    if (heed_abort && m->abort_flag) return false;
-    if (clock64() - t0 > (heed_abort ? m->wait_cycles : kWaitCycles)) break;
-  }
-  give_up(m, status);
-  return false;
-}
 
 // ------------------------------------------------------------------------------------------
 // chunk schedule (identical in every role and every CTA, so no descriptors travel)

@@ -96,9 +96,8 @@ def run_full_size(name, whole, sampled, expect_path=None, check_needle=False):
             out.append(s[0])
         return np.stack(out)
 
-    for l, b, g in sampled:
-        oracle_heads(l, b, [g])
-    for l, b in whole:
+    def compare_whole(l, b):
+        """Every output of one (layer, sequence) against the oracle; returns the oracle's scores."""
         n = cfg.seq_lens[b]
         prefix = n - w
         o_scores = oracle_heads(l, b, range(hkv))
@@ -122,6 +121,12 @@ def run_full_size(name, whole, sampled, expect_path=None, check_needle=False):
         r0, rows = int(g_rowoff[l * B + b]), int(g_hoff[l, b, -1])
         np.testing.assert_array_equal(_bits(plan.k_out[r0:r0 + rows]).cpu().numpy(), ko)
         np.testing.assert_array_equal(_bits(plan.v_out[r0:r0 + rows]).cpu().numpy(), vo)
+        return o_scores
+
+    for l, b, g in sampled:
+        oracle_heads(l, b, [g])
+    for l, b in whole:
+        compare_whole(l, b)
 
     # ---- budgets: the oracle's rule on the device's entropies, bit-exact ---------------------
     for b in range(B):
@@ -133,6 +138,7 @@ def run_full_size(name, whole, sampled, expect_path=None, check_needle=False):
     np.testing.assert_array_equal(g_rowoff, np.concatenate([[0], np.cumsum(g_budget.reshape(-1))]))
 
     # ---- every (layer, sequence): valid top-k, ordered, exact gather --------------------------
+    needle_kept = {}
     for l in range(L):
         for b in range(B):
             n = cfg.seq_lens[b]
@@ -154,7 +160,7 @@ def run_full_size(name, whole, sampled, expect_path=None, check_needle=False):
                     assert int(pos.min()) >= 0 and int(pos.max()) < prefix
                     assert bool((pos[1:] > pos[:-1]).all()), "kept positions must ascend"
                 if needle is not None:
-                    assert bool((pos == needle).any()), "the planted key was evicted"
+                    needle_kept[(l, b, g)] = bool((pos == needle).any())
                 kept[g * prefix + pos] = True
                 rows_all = torch.cat([pos, win_pos]) + tok0[b]
                 o0 = r0 + int(hoff[g])
@@ -168,6 +174,21 @@ def run_full_size(name, whole, sampled, expect_path=None, check_needle=False):
                 tk = kept[ties]
                 n_tk = int(tk.sum())
                 assert bool(tk[:n_tk].all()), "ties must resolve to the lower flat index"
+    if check_needle:
+        # At full length the planted key (logit about 0.9 sqrt(d) = 10) competes with the 1 % of
+        # key rows that are scaled x3 (logits of standard deviation about 4, a hundred and more of
+        # them per head), so a 128-row budget does not always retain it.  Where it is retained
+        # the device and the oracle must agree, and where it is not, too: the decision is checked
+        # against the oracle's own scores and selection on problems of both kinds.
+        lost = list(dict.fromkeys((l, b) for (l, b, g), was_kept in needle_kept.items() if not was_kept))
+        held = list(dict.fromkeys((l, b) for (l, b, g), was_kept in needle_kept.items() if was_kept))
+        for l, b in [x for x in lost if x not in whole][:2] + [x for x in held if x not in whole][:1]:
+            o_scores = compare_whole(l, b)
+            keep_o, _ = O.select_topk(o_scores, int(g_budget[l, b]), w)
+            p = needle_position(cfg, b)
+            for g in range(hkv):
+                assert bool(p in keep_o[g]) == needle_kept[(l, b, g)], (
+                    "device and oracle disagree on the planted key (layer %d seq %d head %d)" % (l, b, g))
     del plan, q, k, v
     torch.cuda.empty_cache()
 
@@ -185,7 +206,7 @@ def test_llama8b_32k_all_layers_in_one_launch():
 
 def test_mistral7b_ragged_all_layers_in_one_launch():
     # w 64 x G 4 = 256 window-query rows per KV head (two units), avg-pool, eight ragged
-    # sequences, a planted key per sequence that every layer must retain
+    # sequences, a planted key per sequence
     cfg = get_config("mistral7b_ragged")
     order = sorted(range(cfg.batch), key=lambda b: cfg.seq_lens[b])
     shortest, longest, middle = order[0], order[-1], order[len(order) // 2]
