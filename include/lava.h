@@ -60,6 +60,7 @@ typedef enum lava_budget_mode { LAVA_BUDGET_DYNAMIC = 0, LAVA_BUDGET_UNIFORM = 1
 #define LAVA_DEV_SHORT_SEQUENCE 1u    /* some sequence has fewer than `window` tokens        */
 #define LAVA_DEV_BUDGET_INFEASIBLE 2u /* total budget outside [L*floor, L*cap]; was clamped  */
 #define LAVA_DEV_WAIT_EXPIRED 4u      /* a bounded wait inside a kernel gave up              */
+#define LAVA_DEV_BAD_SEQLEN 8u        /* some sequence is longer than desc->max_seqlen       */
 
 /* Geometry of one layer (all layers of a model share it).  Plain data, caller-owned (host). */
 typedef struct lava_layer_desc {
@@ -256,9 +257,11 @@ LAVA_API lava_status lava_evict_model_host(const lava_layer_desc* desc, int32_t 
  * call on the hot path reads the environment.  Set them while no call of this library is running.
  *   "select_cluster"     0 = choose by size (default), 8 or 16 CTAs per selection cluster
  *                        (LAVA_SELECT_CLUSTER)
- *   "score_kernel"       0 = choose by geometry (default), 1 = two-pass tensor-core kernel,
- *                        2 = single-pass kernel that keeps the logits in tensor memory where the
- *                        geometry allows it (LAVA_SCORE_KERNEL)
+ *   "score_kernel"       0 or 1 = two-pass tensor-core kernel (default), 2 = single-pass kernel
+ *                        that keeps the exponentials in tensor memory, where the geometry allows
+ *                        it (bf16, d 128, pooling kernel <= 9, about 54K tokens; slower today,
+ *                        and its stored exponentials are fp16: scores within 3e-4 relative)
+ *                        (LAVA_SCORE_KERNEL)
  *   "score_chunk_tiles"  0 = choose per launch, else 1..64 key tiles per chunk of the two-pass
  *                        kernel (LAVA_SM100_CHUNK_TILES)
  *   "score_lead_tiles"   -1 = choose, else extra tiles pass 1 leads pass 2 by (LAVA_SM100_LEAD_TILES)

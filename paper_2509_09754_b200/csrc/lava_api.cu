@@ -152,7 +152,10 @@ Workspace workspace_layout(const lava_layer_desc* d, int n_layers) {
   off = round_up(off + problems * d->n_kv_heads * w.n_slices * sizeof(double2), 256);
   w.off_sm100 = off;
   Geom g;
-  if (make_geom(d, &g) == LAVA_OK && sm100_supported(g)) off += sm100_layout(g, n_layers).total;
+  const bool tensor_path = make_geom(d, &g) == LAVA_OK && sm100_supported(g);
+  if (tensor_path) off += sm100_layout(g, n_layers).total;
+  w.off_tmem = off;
+  if (tensor_path && tmem_supported(g)) off += tmem_layout(g, n_layers).total;
   w.total = off;
   return w;
 }
@@ -264,10 +267,18 @@ lava_status lava_score_layers(const lava_layer_desc* desc, int32_t n_layers, con
     return fail(LAVA_ERR_WORKSPACE, "workspace too small: %zu < %zu bytes", workspace_bytes,
                 lay.total);
   if (!aligned16(workspace)) return fail(LAVA_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
-  if (sm100_supported(g) && !options().force_generic)
+  if (sm100_supported(g) && !options().force_generic) {
+    // the single-pass kernel (exponentials kept in tensor memory) is opt-in: the exchange of row
+    // statistics between the CTAs outlasts what six exponent buffers can cover, so it is the
+    // slower of the two today
+    if (options().score_kernel == 2 && tmem_supported(g) && tmem_fits(g, tmem_grid(g, n_layers)))
+      return launch_score_tmem(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
+                               v_layer_stride, vbar_in, scores, vbar_out, entropy,
+                               (char*)workspace, lay.off_tmem, (cudaStream_t)stream);
     return launch_score_sm100(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
                               v_layer_stride, vbar_in, scores, vbar_out, entropy,
                               (char*)workspace, lay.off_sm100, (cudaStream_t)stream);
+  }
   return launch_score_generic(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
                               v_layer_stride, vbar_in, scores, vbar_out, entropy,
                               (char*)workspace, lay, (cudaStream_t)stream);

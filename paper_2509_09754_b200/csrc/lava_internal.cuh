@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of liblava (not part of the C ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -48,7 +49,7 @@ struct Workspace {
   static constexpr size_t kStatusBytes = 256;
   static constexpr int kSlice = 512;    // keys per block in the generic score kernels
   static constexpr int kVSlice = 1024;  // V rows per block in the value-norm kernel
-  size_t off_vpart, off_stats, off_lse, off_vbar, off_ent, off_sm100, total;
+  size_t off_vpart, off_stats, off_lse, off_vbar, off_ent, off_sm100, off_tmem, total;
   int n_slices, n_vslices;
 };
 Workspace workspace_layout(const lava_layer_desc* d, int n_layers);
@@ -91,6 +92,25 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
                                const void* v, long long q_ls, long long k_ls, long long v_ls,
                                const float* vbar_in, float* scores, float* vbar_out,
                                double* entropy, char* ws_base, size_t ws_off, cudaStream_t stream);
+// Tensor maps of the query window ([layer][batch*H_q*w rows][128]) and of K
+// ([layer][H_kv][tokens][128]) in boxes of 64 x 128 bf16 elements with the 128-byte swizzle.
+lava_status encode_score_maps(const Geom& g, int n_layers, const void* q, const void* k,
+                              long long q_ls, long long k_ls, CUtensorMap* map_q,
+                              CUtensorMap* map_k);
+// Single-pass Blackwell score path (logits and exponentials stay in tensor memory).
+struct TmemLayout {
+  int ok, nunit, tmax, kfold, gmax, heads_total, units_total;
+  long long kjobs_cap;
+  size_t off_sync, sync_bytes, off_part, off_gpart, off_ent, total;
+};
+bool tmem_supported(const Geom& g);
+bool tmem_fits(const Geom& g, int grid);
+int tmem_grid(const Geom& g, int n_layers);
+TmemLayout tmem_layout(const Geom& g, int n_layers);
+lava_status launch_score_tmem(const Geom& g, int n_layers, const void* q, const void* k,
+                              const void* v, long long q_ls, long long k_ls, long long v_ls,
+                              const float* vbar_in, float* scores, float* vbar_out,
+                              double* entropy, char* ws_base, size_t ws_off, cudaStream_t stream);
 lava_status launch_wo_norm(const void* w_o, int dtype, long long rows, long long cols,
                            float* out, cudaStream_t stream);
 lava_status launch_budgets(int n_layers, int batch, const double* entropy,

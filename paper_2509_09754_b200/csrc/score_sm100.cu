@@ -1112,17 +1112,14 @@ Sm100Layout sm100_layout(const Geom& g, int n_layers) {
   return l;
 }
 
-lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const void* k,
-                               const void* v, long long q_ls, long long k_ls, long long v_ls,
-                               const float* vbar_in, float* scores, float* vbar_out,
-                               double* entropy, char* ws_base, size_t ws_off, cudaStream_t stream) {
-  char* ws = ws_base + ws_off;
+lava_status encode_score_maps(const Geom& g, int n_layers, const void* q, const void* k,
+                              long long q_ls, long long k_ls, CUtensorMap* map_q_out,
+                              CUtensorMap* map_k_out) {
   EncodeTiledFn encode = encode_fn();
   if (!encode) return fail(LAVA_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
-  const Sm100Layout lay = sm100_layout(g, n_layers);
-
+  CUtensorMap& map_q = *map_q_out;
+  CUtensorMap& map_k = *map_k_out;
   // Q: [layer][batch*H_q*w rows][128]; K: [layer][H_kv][tokens][128]; boxes of 64 x 128 elements
-  CUtensorMap map_q, map_k;
   {
     const cuuint64_t rows = (cuuint64_t)g.batch * g.n_q_heads * g.window;
     const cuuint64_t dims[3] = {128, rows, (cuuint64_t)n_layers};
@@ -1146,6 +1143,22 @@ lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const
                es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return fail(LAVA_ERR_CUDA, "tensor map for K could not be encoded");
+  }
+
+  return LAVA_OK;
+}
+
+lava_status launch_score_sm100(const Geom& g, int n_layers, const void* q, const void* k,
+                               const void* v, long long q_ls, long long k_ls, long long v_ls,
+                               const float* vbar_in, float* scores, float* vbar_out,
+                               double* entropy, char* ws_base, size_t ws_off, cudaStream_t stream) {
+  char* ws = ws_base + ws_off;
+  const Sm100Layout lay = sm100_layout(g, n_layers);
+
+  CUtensorMap map_q, map_k;
+  {
+    const lava_status mrc = encode_score_maps(g, n_layers, q, k, q_ls, k_ls, &map_q, &map_k);
+    if (mrc != LAVA_OK) return mrc;
   }
 
   const int sms = sm_count();

@@ -235,3 +235,24 @@ def test_split_query_groups(kw):
     assert lava.lava_score_path(desc) == 2, "this geometry must run as two units per KV head"
     compare_eviction(cfg)
 
+
+
+@pytest.mark.parametrize("kw", [
+    dict(seq_lens=(1733,), n_layers=3, budget_per_head=160),                              # G 4 x w 32
+    dict(seq_lens=(777, 1290, 515), n_layers=2, budget_per_head=128, window=64,
+         pool_kind=lava.LAVA_POOL_AVG, pool_kernel=5),                                    # two units, avg-pool, ragged
+    dict(seq_lens=(2100,), n_layers=2, budget_per_head=200, n_q_heads=14, n_kv_heads=2),  # G 7: units of 4 and 3
+    dict(seq_lens=(900,), n_layers=2, budget_per_head=64, n_q_heads=32, n_kv_heads=2, window=16),  # 8 heads per unit
+    dict(seq_lens=(1300,), n_layers=1, budget_per_head=140, n_q_heads=4, n_kv_heads=2, window=128),
+    dict(seq_lens=(33, 64), n_layers=2, budget_per_head=33),                              # one candidate / n == 2w
+])
+def test_single_pass_score_kernel(kw):
+    """The opt-in single-pass kernel (exponentials kept in tensor memory as fp16) against the
+    oracle on the geometries it covers, whole eviction."""
+    cfg = get_config("llama8b_8k").scaled(**kw)
+    lava.lava_set_option("score_kernel", 2)
+    try:
+        rep = compare_eviction(cfg)
+        assert rep["max_rel_err"] < 1e-3
+    finally:
+        lava.lava_set_option("score_kernel", 0)
