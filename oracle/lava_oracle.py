@@ -37,7 +37,8 @@ import math
 import numpy as np
 
 POOL_NONE, POOL_MAX, POOL_AVG = 0, 1, 2
-BUDGET_DYNAMIC, BUDGET_UNIFORM = 0, 1
+BUDGET_DYNAMIC, BUDGET_UNIFORM, BUDGET_PYRAMID = 0, 1, 2
+VALUE_NORM_MAX, VALUE_NORM_UNIT, VALUE_NORM_TOKEN = 0, 1, 2
 
 
 # --------------------------------------------------------------------------------------------
@@ -116,6 +117,45 @@ def value_norm(v):
 # --------------------------------------------------------------------------------------------
 # Step 5: LAVa score with GQA group maximum (Definition 1; Sec. 4.3)
 # --------------------------------------------------------------------------------------------
+def token_value_norms(v):
+    """Row L1 norms ||V_g[i]||_1 of every cached position: [H_kv, n] (the VATP weight)."""
+    return np.abs(np.asarray(v, dtype=np.float64)).sum(axis=2)
+
+
+def variant_scores(q_win, k, v, w, pool_kind=POOL_MAX, pool_kernel=7, sm_scale=None,
+                   c_hat=1.0, value_term=VALUE_NORM_MAX):
+    """The score with the value term of the methods the paper compares against (its table of
+    score functions and the related-work paragraph on VATP):
+
+    VALUE_NORM_MAX    LAVa, Definition 1: the head's largest row L1 norm (same as lava_scores)
+    VALUE_NORM_UNIT   SnapKV / AdaKV: the pooled window-mean attention alone (value term 1)
+    VALUE_NORM_TOKEN  VATP: every position weighted by its own ||V_g[i]||_1
+    In all three the pooled window mean of each query head is weighted first and the group
+    maximum (Sec. 4.3) is taken last.  Returns [H_kv, P].
+    """
+    q_win = np.asarray(q_win, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    n_q_heads = q_win.shape[0]
+    n_kv_heads, n, _ = k.shape
+    group = n_q_heads // n_kv_heads
+    prefix = n - w
+    att = window_attention(q_win, k, sm_scale)
+    pooled = pool1d(window_mean_prefix(att, w), pool_kind, pool_kernel)      # [H_q, P]
+    if value_term == VALUE_NORM_MAX:
+        weight = np.repeat(value_norm(v)[:, None], prefix, axis=1)
+    elif value_term == VALUE_NORM_UNIT:
+        weight = np.ones((n_kv_heads, prefix))
+    elif value_term == VALUE_NORM_TOKEN:
+        weight = token_value_norms(v)[:, :prefix]
+    else:
+        raise ValueError("unknown value-norm variant")
+    scores = np.empty((n_kv_heads, prefix), dtype=np.float64)
+    for g in range(n_kv_heads):
+        scaled = float(c_hat) * weight[g][None, :] * pooled[g * group:(g + 1) * group]
+        scores[g] = scaled.max(axis=0)
+    return scores
+
+
 def lava_scores(q_win, k, v, w, pool_kind=POOL_MAX, pool_kernel=7, sm_scale=None,
                 c_hat=1.0, vbar=None):
     """s_g[i] = c_hat * Vbar_g * max_{h in group g} pool(a_h)[i], i < P.  Returns [H_kv, P]."""
@@ -177,13 +217,28 @@ def _largest_remainder(shares, total):
     return base
 
 
-def layer_budgets(entropy, total_budget, lo, hi, mode=BUDGET_DYNAMIC):
+def pyramid_weights(n_layers, beta=20.0):
+    """Relative layer budgets of the PyramidKV rule the paper quotes (its paragraph on
+    PyramidKV): B_{L-1} = B / (beta L), B_0 = 2 B / L - B_{L-1}, and a straight line between
+    them, descending with depth (the printed interpolation has its sign garbled; the line from
+    B_0 at layer 0 to B_{L-1} at the last layer is what "like a pyramid" describes).  Returned
+    for B = 1; the weights are positive and sum to 1."""
+    n_layers = int(n_layers)
+    if n_layers == 1:
+        return [1.0]
+    last = 1.0 / (float(beta) * n_layers)
+    first = 2.0 / n_layers - last
+    return [first + (last - first) * l / (n_layers - 1) for l in range(n_layers)]
+
+
+def layer_budgets(entropy, total_budget, lo, hi, mode=BUDGET_DYNAMIC, beta=20.0):
     """Integer layer budgets with sum == total_budget and lo <= B_l <= hi.
 
     entropy      : [L] layer uncertainties e_l
     total_budget : the model-wide budget (KV-head entries, window rows included)
     lo, hi       : per-layer floor (H_kv*w: the window is always kept) and cap (H_kv*n)
-    mode         : BUDGET_DYNAMIC -> shares e_l / sum e ; BUDGET_UNIFORM -> equal shares
+    mode         : BUDGET_DYNAMIC -> shares e_l / sum e ; BUDGET_UNIFORM -> equal shares ;
+                   BUDGET_PYRAMID -> shares pyramid_weights(L, beta) (the entropies are ignored)
 
     Rule.  Layers start "active".  Each round the remaining budget R (total minus what clamped
     layers hold) is shared among active layers in proportion to e_l (equally if their e sum to
@@ -195,6 +250,8 @@ def layer_budgets(entropy, total_budget, lo, hi, mode=BUDGET_DYNAMIC):
     """
     e = [float(x) for x in entropy]
     n_layers = len(e)
+    if mode == BUDGET_PYRAMID:
+        e = pyramid_weights(n_layers, beta)
     total_budget, lo, hi = int(total_budget), int(lo), int(hi)
     if not (n_layers * lo <= total_budget <= n_layers * hi):
         raise ValueError("infeasible budget: need L*lo <= total <= L*hi")
@@ -266,6 +323,29 @@ def select_topk(scores, layer_budget, w):
 # --------------------------------------------------------------------------------------------
 # Step 9: compaction (Algorithm 1: K-hat = K (.) I, V-hat = V (.) I, physically a gather)
 # --------------------------------------------------------------------------------------------
+def select_topk_per_head(scores, layer_budget, w):
+    """The paper's "- head dynamic" ablation (Sec. 5.4): the layer budget is split evenly over
+    the heads and every head keeps its own best entries, with no comparison across heads.
+
+    The ``layer_budget - H_kv*w`` selectable entries are shared as evenly as integers allow (the
+    first ``remainder`` heads get one more); a head with fewer candidates than its share keeps
+    all of them (the surplus is not handed on: budgets are fixed).  Same return as select_topk.
+    """
+    s = np.asarray(scores, dtype=np.float64)
+    n_kv_heads, prefix = s.shape
+    k_sel = max(0, int(layer_budget) - n_kv_heads * int(w))
+    base, extra = divmod(k_sel, n_kv_heads)
+    keep = []
+    for g in range(n_kv_heads):
+        k_g = min(prefix, base + (1 if g < extra else 0))
+        one, _ = select_topk(s[g:g + 1], k_g + int(w), w)        # the layer-wide rule on one head
+        keep.append(one[0])
+    head_offsets = np.zeros(n_kv_heads + 1, dtype=np.int64)
+    for g in range(n_kv_heads):
+        head_offsets[g + 1] = head_offsets[g] + len(keep[g]) + int(w)
+    return keep, head_offsets
+
+
 def compact_kv(k, v, keep, w):
     """Rows of every head in temporal order: kept prefix rows, then the w window rows.
 

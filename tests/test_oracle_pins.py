@@ -453,3 +453,83 @@ def test_model_level_invariants():
             np.testing.assert_array_equal(rows, ks[l][g][pos])
     uni = O.evict_model(qs, ks, vs, w, total, O.POOL_MAX, 7, mode=O.BUDGET_UNIFORM)
     assert uni["budgets"] == [31, 31, 31]
+
+
+# ---------------------------------------------------------------- ablation modes (Sec. 5.4; table of methods)
+def test_per_head_selection_is_the_layer_rule_on_each_head_alone():
+    """"- head dynamic": every head keeps its own share; with one head the two rules coincide,
+    and a head's choice never depends on the other heads' scores."""
+    rng = np.random.RandomState(41)
+    hkv, prefix, w = 3, 40, 4
+    s = rng.rand(hkv, prefix)
+    one, off1 = O.select_topk_per_head(s[:1], w + 13, w)
+    ref, off2 = O.select_topk(s[:1], w + 13, w)
+    np.testing.assert_array_equal(one[0], ref[0])
+    np.testing.assert_array_equal(off1, off2)
+    budget = hkv * w + 20                                    # 20 = 3 * 6 + 2: shares 7, 7, 6
+    keep, off = O.select_topk_per_head(s, budget, w)
+    assert [len(x) for x in keep] == [7, 7, 6]
+    np.testing.assert_array_equal(off, [0, 11, 22, 32])
+    for g in range(hkv):
+        np.testing.assert_array_equal(np.sort(keep[g]), keep[g])
+        want = np.sort(np.argsort(-s[g], kind="stable")[:len(keep[g])])
+        np.testing.assert_array_equal(keep[g], want)
+    s2 = s.copy()
+    s2[1] *= 1000.0                                          # another head's scale changes nothing
+    keep2, _ = O.select_topk_per_head(s2, budget, w)
+    for g in range(hkv):
+        np.testing.assert_array_equal(keep2[g], keep[g])
+    # a head with fewer candidates than its share keeps all of them; the rest is not handed on
+    keep3, off3 = O.select_topk_per_head(s[:, :5], hkv * w + 20, w)
+    assert [len(x) for x in keep3] == [5, 5, 5] and off3[-1] == hkv * (5 + w)
+    # layer-wide selection of the same budget differs once one head dominates
+    wide, _ = O.select_topk(s2, budget, w)
+    assert len(wide[1]) == 20 and len(wide[0]) == 0
+
+
+def test_pyramid_weights_follow_the_quoted_rule():
+    """PyramidKV paragraph: B_{L-1} = B/(beta L), B_0 = 2B/L - B_{L-1}, a straight line between."""
+    for n_layers, beta in ((32, 20.0), (5, 2.0), (2, 4.0)):
+        wts = O.pyramid_weights(n_layers, beta)
+        assert sum(wts) == pytest.approx(1.0, abs=1e-12)
+        assert wts[-1] == pytest.approx(1.0 / (beta * n_layers), abs=1e-15)
+        assert wts[0] == pytest.approx(2.0 / n_layers - 1.0 / (beta * n_layers), abs=1e-15)
+        steps = np.diff(wts)
+        assert np.all(steps < 0) and np.allclose(steps, steps[0], atol=1e-15)
+    assert O.pyramid_weights(1) == [1.0]
+    # hand-worked: L = 4, beta = 2, B = 800 -> B_3 = 100, B_0 = 300, line 300, 233.33, 166.67, 100
+    want = O.layer_budgets([0.0] * 4, 800, 0, 10_000, O.BUDGET_PYRAMID, beta=2.0)
+    assert want == [300, 233, 167, 100]
+    # the entropies play no part, the floor still binds (the last layer is lifted to it)
+    assert O.layer_budgets([9.0, 1.0, 5.0, 2.0], 800, 0, 10_000, O.BUDGET_PYRAMID, beta=2.0) == want
+    clamped = O.layer_budgets([0.0] * 4, 800, 150, 10_000, O.BUDGET_PYRAMID, beta=2.0)
+    assert clamped[-1] == 150 and sum(clamped) == 800 and clamped[0] > clamped[1] > clamped[2] >= 150
+
+
+def test_value_term_variants():
+    """VALUE_NORM_MAX is Definition 1; UNIT is the pooled window mean alone (the SnapKV / AdaKV
+    score of the paper's table); TOKEN weights position i by ||V[i]||_1 (VATP)."""
+    hq, hkv, n, w, d = 4, 2, 30, 4, 8
+    q, k, v = _rand_layer(51, hq, hkv, n, w, d, vscale=[1.0, 3.0])
+    base = O.lava_scores(q, k, v, w, O.POOL_MAX, 5)
+    np.testing.assert_array_equal(O.variant_scores(q, k, v, w, O.POOL_MAX, 5), base)
+    unit = O.variant_scores(q, k, v, w, O.POOL_MAX, 5, value_term=O.VALUE_NORM_UNIT)
+    vbar = O.value_norm(v)
+    np.testing.assert_allclose(unit * vbar[:, None], base, rtol=1e-13)
+    # unit scores are pooled window means: with max-pool 1 each head's row sums to at most 1
+    plain = O.variant_scores(q, k, v, w, O.POOL_NONE, 1, value_term=O.VALUE_NORM_UNIT)
+    att = O.window_attention(q, k)
+    a = O.window_mean_prefix(att, w)
+    np.testing.assert_allclose(plain, np.maximum(a[0::2], a[1::2]), rtol=1e-13)
+    # per-token weights: with rows of V of equal norm c the score is c times the unit score;
+    # scaling ONE row of V scales only that position's score (no pooling), unlike Vbar
+    v_eq = np.sign(v) * 0.5
+    tok = O.variant_scores(q, k, v_eq, w, O.POOL_NONE, 1, value_term=O.VALUE_NORM_TOKEN)
+    np.testing.assert_allclose(tok, 0.5 * d * plain, rtol=1e-13)
+    v_one = v_eq.copy()
+    v_one[1, 7] *= 10.0
+    tok2 = O.variant_scores(q, k, v_one, w, O.POOL_NONE, 1, value_term=O.VALUE_NORM_TOKEN)
+    np.testing.assert_allclose(tok2[1, 7], 10.0 * tok[1, 7], rtol=1e-13)
+    tok2[1, 7] = tok[1, 7]
+    np.testing.assert_array_equal(tok2, tok)
+    np.testing.assert_allclose(O.token_value_norms(v_one)[1, 7], 5.0 * d, rtol=1e-13)
