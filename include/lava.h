@@ -54,13 +54,28 @@ typedef enum lava_status {
 
 typedef enum lava_dtype { LAVA_F32 = 0, LAVA_BF16 = 1 } lava_dtype;
 typedef enum lava_pool { LAVA_POOL_NONE = 0, LAVA_POOL_MAX = 1, LAVA_POOL_AVG = 2 } lava_pool;
-typedef enum lava_budget_mode { LAVA_BUDGET_DYNAMIC = 0, LAVA_BUDGET_UNIFORM = 1 } lava_budget_mode;
+typedef enum lava_budget_mode {
+  LAVA_BUDGET_DYNAMIC = 0,  /* Algorithm 2: shares e_l / sum e                                   */
+  LAVA_BUDGET_UNIFORM = 1,  /* "- layer dynamic" / LAVa-Uniform of the ablation (Sec. 5.4): B / L   */
+  LAVA_BUDGET_PYRAMID = 2   /* LAVa-Pyramid of the layer-allocation comparison: the PyramidKV line
+                               B_{L-1} = B / (beta L), B_0 = 2B/L - B_{L-1}, descending with depth;
+                               beta = mode >> 8 (0 means 20): pass LAVA_BUDGET_PYRAMID | beta << 8   */
+} lava_budget_mode;
 
 /* Bits of the device status word. */
 #define LAVA_DEV_SHORT_SEQUENCE 1u    /* some sequence has fewer than `window` tokens        */
 #define LAVA_DEV_BUDGET_INFEASIBLE 2u /* total budget outside [L*floor, L*cap]; was clamped  */
 #define LAVA_DEV_WAIT_EXPIRED 4u      /* a bounded wait inside a kernel gave up              */
 #define LAVA_DEV_BAD_SEQLEN 8u        /* some sequence is longer than desc->max_seqlen       */
+
+/* Variants of the method (the ablation of Sec. 5.4 and the score functions of the methods the
+ * paper compares with).  0 is LAVa as published. */
+#define LAVA_FLAG_PER_HEAD_TOPK 1u    /* "- head dynamic": every KV head keeps its even share of the
+                                         layer budget, no comparison across heads (lava_select_topk) */
+#define LAVA_FLAG_UNIT_VALUE_NORM 2u  /* SnapKV / AdaKV score: value term 1 instead of Vbar; V is not
+                                         read and may be NULL (lava_score_layer)                     */
+#define LAVA_FLAG_TOKEN_VALUE_NORM 4u /* VATP score: ||V_g[i]||_1 of every position instead of Vbar
+                                         (lava_score_layer; vbar_in must be NULL)                    */
 
 /* Geometry of one layer (all layers of a model share it).  Plain data, caller-owned (host). */
 typedef struct lava_layer_desc {
@@ -73,7 +88,7 @@ typedef struct lava_layer_desc {
   int32_t dtype;       /* lava_dtype of Q, K, V and of the compacted output                 */
   int32_t batch;       /* number of sequences (>= 1)                                        */
   int32_t max_seqlen;  /* upper bound on any sequence length (0 => total_tokens)            */
-  int32_t reserved;    /* must be 0                                                         */
+  int32_t flags;       /* LAVA_FLAG_* bits, 0 for the paper's method                        */
   const int32_t* cu_seqlens; /* device int32 [batch+1] token offsets; NULL => batch == 1    */
   int64_t total_tokens;      /* sum of sequence lengths                                     */
   int64_t k_stride_head, k_stride_tok; /* K[g][tok][c] = k[g*k_stride_head + tok*k_stride_tok + c] */
@@ -167,7 +182,7 @@ LAVA_API lava_status lava_score_layer_static(const lava_layer_desc* desc, const 
  *   total_budget     int64 [batch]: model-wide budget of each sequence in KV-head rows,
  *                    window rows included
  *   floor_per_layer  int64 [batch]: H_kv * w      cap_per_layer  int64 [batch]: H_kv * n_b
- *   mode             lava_budget_mode (uniform = total/L per layer, the paper's ablation)
+ *   mode             lava_budget_mode (uniform and pyramid ignore the entropies)
  *   layer_budget     out int64 [n_layers, batch], sums to total_budget[b] over layers
  *   layer_row_offset out int64 [n_layers*batch + 1]: exclusive prefix sums of layer_budget in
  *                    (layer, sequence) order = first row of each (layer, sequence) in the

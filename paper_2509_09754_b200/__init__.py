@@ -6,7 +6,8 @@ kernels.  There is no CPU or PyTorch fallback; a missing library raises at first
 """
 from .binding import (  # noqa: F401
     LAVA_BF16, LAVA_F32, LAVA_POOL_AVG, LAVA_POOL_MAX, LAVA_POOL_NONE,
-    LAVA_BUDGET_DYNAMIC, LAVA_BUDGET_UNIFORM,
+    LAVA_BUDGET_DYNAMIC, LAVA_BUDGET_UNIFORM, LAVA_BUDGET_PYRAMID,
+    LAVA_FLAG_PER_HEAD_TOPK, LAVA_FLAG_UNIT_VALUE_NORM, LAVA_FLAG_TOKEN_VALUE_NORM,
     LavaError, LayerDesc, library_path, load_library,
     lava_version, lava_last_error, lava_workspace_bytes, lava_poll_status, lava_wo_norm,
     lava_score_layer, lava_score_layer_static, lava_score_layers, lava_layer_budgets,

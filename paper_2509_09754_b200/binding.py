@@ -10,7 +10,8 @@ import torch
 
 LAVA_F32, LAVA_BF16 = 0, 1
 LAVA_POOL_NONE, LAVA_POOL_MAX, LAVA_POOL_AVG = 0, 1, 2
-LAVA_BUDGET_DYNAMIC, LAVA_BUDGET_UNIFORM = 0, 1
+LAVA_BUDGET_DYNAMIC, LAVA_BUDGET_UNIFORM, LAVA_BUDGET_PYRAMID = 0, 1, 2
+LAVA_FLAG_PER_HEAD_TOPK, LAVA_FLAG_UNIT_VALUE_NORM, LAVA_FLAG_TOKEN_VALUE_NORM = 1, 2, 4
 
 _STATUS_NAMES = {0: "LAVA_OK", 1: "LAVA_ERR_INVALID_ARG", 2: "LAVA_ERR_UNSUPPORTED",
                  3: "LAVA_ERR_WORKSPACE", 4: "LAVA_ERR_CUDA", 5: "LAVA_ERR_TIMEOUT"}
@@ -28,7 +29,7 @@ class _CDesc(ctypes.Structure):
         ("head_dim", ctypes.c_int32), ("window", ctypes.c_int32),
         ("pool_kind", ctypes.c_int32), ("pool_kernel", ctypes.c_int32),
         ("dtype", ctypes.c_int32), ("batch", ctypes.c_int32),
-        ("max_seqlen", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("max_seqlen", ctypes.c_int32), ("flags", ctypes.c_int32),
         ("cu_seqlens", ctypes.c_void_p), ("total_tokens", ctypes.c_int64),
         ("k_stride_head", ctypes.c_int64), ("k_stride_tok", ctypes.c_int64),
         ("v_stride_head", ctypes.c_int64), ("v_stride_tok", ctypes.c_int64),
@@ -135,12 +136,13 @@ class LayerDesc:
     v_stride_tok: int = 0
     sm_scale: float = 0.0
     c_hat: float = 0.0
+    flags: int = 0
 
     @staticmethod
     def for_tensors(q_win: torch.Tensor, k: torch.Tensor, v: Optional[torch.Tensor], window: int,
                     pool_kind: int = LAVA_POOL_MAX, pool_kernel: int = 7,
                     cu_seqlens: Optional[torch.Tensor] = None, max_seqlen: int = 0,
-                    sm_scale: float = 0.0, c_hat: float = 0.0) -> "LayerDesc":
+                    sm_scale: float = 0.0, c_hat: float = 0.0, flags: int = 0) -> "LayerDesc":
         """q_win [batch, H_q, w, d]; k, v [H_kv, total_tokens, d] (one layer's views)."""
         batch, hq, w, d = q_win.shape
         hkv, total, _ = k.shape
@@ -150,7 +152,7 @@ class LayerDesc:
             pool_kernel=pool_kernel, dtype=_dtype_code(k), batch=batch, max_seqlen=max_seqlen,
             cu_seqlens=cu_seqlens, total_tokens=total, k_stride_head=k.stride(0),
             k_stride_tok=k.stride(1), v_stride_head=vv.stride(0), v_stride_tok=vv.stride(1),
-            sm_scale=sm_scale, c_hat=c_hat)
+            sm_scale=sm_scale, c_hat=c_hat, flags=flags)
 
     @property
     def total_scores(self) -> int:
@@ -158,7 +160,7 @@ class LayerDesc:
 
     def to_c(self) -> _CDesc:
         return _CDesc(self.n_q_heads, self.n_kv_heads, self.head_dim, self.window, self.pool_kind,
-                      self.pool_kernel, self.dtype, self.batch, self.max_seqlen, 0,
+                      self.pool_kernel, self.dtype, self.batch, self.max_seqlen, self.flags,
                       None if self.cu_seqlens is None else self.cu_seqlens.data_ptr(),
                       self.total_tokens, self.k_stride_head, self.k_stride_tok,
                       self.v_stride_head, self.v_stride_tok, self.sm_scale, self.c_hat)

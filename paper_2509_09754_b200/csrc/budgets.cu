@@ -4,7 +4,8 @@
 // fused multiply-add) and layer-ordered sums, so the integers depend only on the entropies
 // given.  Rule:
 //   * active layers share the remaining budget R in proportion to e_l (equally when the sum of
-//     their e is zero / not finite, or in uniform mode);
+//     their e is zero / not finite, or in uniform mode; in pyramid mode e_l is replaced by the
+//     PyramidKV line quoted in the paper's layer-allocation comparison);
 //   * shares become integers by largest remainder: floors first, then +1 in order of
 //     decreasing fractional part, ties to the lower layer;
 //   * if some active layer falls below the floor or above the cap, the total shortfall and
@@ -38,8 +39,21 @@ budgets_kernel(int n_layers, int batch, const double* entropy, const long long* 
     if (status && l == 0) atomicOr(status, LAVA_DEV_BUDGET_INFEASIBLE);
     tot = tot < (long long)n_layers * lo ? (long long)n_layers * lo : (long long)n_layers * hi;
   }
+  const int kind = mode & 0xff;
   if (l < n_layers) {
-    sh_e[l] = entropy[(size_t)l * batch + b];
+    double e = entropy[(size_t)l * batch + b];
+    if (kind == LAVA_BUDGET_PYRAMID) {
+      // the PyramidKV line the paper quotes, for a total of 1: last = 1 / (beta L),
+      // first = 2 / L - last, straight in between (same operations, same order, as double)
+      const double beta = (mode >> 8) > 0 ? (double)(mode >> 8) : 20.0;
+      const double nl = (double)n_layers;
+      const double last = __ddiv_rn(1.0, __dmul_rn(beta, nl));
+      const double first = __dsub_rn(__ddiv_rn(2.0, nl), last);
+      e = n_layers == 1 ? 1.0
+                        : __dadd_rn(first, __ddiv_rn(__dmul_rn(__dsub_rn(last, first), (double)l),
+                                                     (double)(n_layers - 1)));
+    }
+    sh_e[l] = e;
     sh_active[l] = 1;
     sh_val[l] = 0;
   }
@@ -56,7 +70,7 @@ budgets_kernel(int n_layers, int batch, const double* entropy, const long long* 
       for (int m = 0; m < n_layers; ++m)
         if (sh_active[m]) esum = __dadd_rn(esum, sh_e[m]);
       sh_esum = esum;
-      sh_uniform = (mode == LAVA_BUDGET_UNIFORM) || !(esum > 0.0) || isinf(esum) || isnan(esum);
+      sh_uniform = (kind == LAVA_BUDGET_UNIFORM) || !(esum > 0.0) || isinf(esum) || isnan(esum);
     }
     __syncthreads();
     const bool active = l < n_layers && sh_active[l];

@@ -87,7 +87,9 @@ lava_status make_geom(const lava_layer_desc* d, Geom* out) {
   if (d->batch < 1) return fail(LAVA_ERR_INVALID_ARG, "batch must be >= 1");
   if (d->batch > 1 && !d->cu_seqlens)
     return fail(LAVA_ERR_INVALID_ARG, "cu_seqlens is required when batch > 1");
-  if (d->reserved != 0) return fail(LAVA_ERR_INVALID_ARG, "reserved must be 0");
+  if (d->flags < 0 || d->flags > 7) return fail(LAVA_ERR_INVALID_ARG, "unknown bits in flags");
+  if ((d->flags & LAVA_FLAG_UNIT_VALUE_NORM) && (d->flags & LAVA_FLAG_TOKEN_VALUE_NORM))
+    return fail(LAVA_ERR_INVALID_ARG, "the unit and the per-token value term exclude each other");
   if (d->total_tokens < (int64_t)d->batch * d->window)
     return fail(LAVA_ERR_INVALID_ARG, "total_tokens (%lld) < batch*window: every sequence needs "
                 "at least `window` tokens", (long long)d->total_tokens);
@@ -119,6 +121,7 @@ lava_status make_geom(const lava_layer_desc* d, Geom* out) {
   g.dtype = d->dtype;
   g.batch = d->batch;
   g.max_seqlen = d->max_seqlen > 0 ? d->max_seqlen : (int)d->total_tokens;
+  g.flags = d->flags;
   g.cu_seqlens = d->cu_seqlens;
   g.total_tokens = d->total_tokens;
   g.total_scores = (long long)d->n_kv_heads * (d->total_tokens - (long long)d->batch * d->window);
@@ -147,6 +150,8 @@ Workspace workspace_layout(const lava_layer_desc* d, int n_layers) {
   w.off_lse = off;
   off = round_up(off + problems * d->n_q_heads * d->window * sizeof(float), 256);
   w.off_vbar = off;
+  off = round_up(off + problems * d->n_kv_heads * sizeof(float), 256);
+  w.off_ones = off;
   off = round_up(off + problems * d->n_kv_heads * sizeof(float), 256);
   w.off_ent = off;
   off = round_up(off + problems * d->n_kv_heads * w.n_slices * sizeof(double2), 256);
@@ -255,7 +260,13 @@ lava_status lava_score_layers(const lava_layer_desc* desc, int32_t n_layers, con
   if (n_layers < 1) return fail(LAVA_ERR_INVALID_ARG, "n_layers must be >= 1");
   if (!q_win || !k || !entropy || (!scores && g.total_scores > 0))
     return fail(LAVA_ERR_INVALID_ARG, "q_win, k, scores and entropy are required");
-  if (!v && !vbar_in) return fail(LAVA_ERR_INVALID_ARG, "v may be NULL only if vbar_in is given");
+  const bool unit_term = (g.flags & (LAVA_FLAG_UNIT_VALUE_NORM | LAVA_FLAG_TOKEN_VALUE_NORM)) != 0;
+  const bool token_term = (g.flags & LAVA_FLAG_TOKEN_VALUE_NORM) != 0;
+  if (!v && !vbar_in && !(unit_term && !token_term))
+    return fail(LAVA_ERR_INVALID_ARG, "v may be NULL only if vbar_in is given");
+  if (unit_term && vbar_in)
+    return fail(LAVA_ERR_INVALID_ARG, "vbar_in must be NULL with a value-term flag");
+  if (token_term && !v) return fail(LAVA_ERR_INVALID_ARG, "the per-token value term needs v");
   if (!aligned16(q_win) || !aligned16(k) || (v && !aligned16(v)) || !aligned16(scores))
     return fail(LAVA_ERR_INVALID_ARG, "q_win, k, v and scores must be 16-byte aligned");
   if (n_layers > 1 && (q_layer_stride % 8 || k_layer_stride % 8 || v_layer_stride % 8 ||
@@ -267,21 +278,38 @@ lava_status lava_score_layers(const lava_layer_desc* desc, int32_t n_layers, con
     return fail(LAVA_ERR_WORKSPACE, "workspace too small: %zu < %zu bytes", workspace_bytes,
                 lay.total);
   if (!aligned16(workspace)) return fail(LAVA_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
+  cudaStream_t st = (cudaStream_t)stream;
+  const void* v_used = v;
+  if (unit_term) {
+    // the score kernels run with a value-norm array of ones and never touch V
+    float* ones = reinterpret_cast<float*>((char*)workspace + lay.off_ones);
+    rc = launch_fill_ones(ones, (long long)n_layers * g.batch * g.n_kv_heads, st);
+    if (rc != LAVA_OK) return rc;
+    vbar_in = ones;
+    v_used = nullptr;
+  }
   if (sm100_supported(g) && !options().force_generic) {
     // the single-pass kernel (exponentials kept in tensor memory) is opt-in: the exchange of row
     // statistics between the CTAs outlasts what six exponent buffers can cover, so it is the
     // slower of the two today
     if (options().score_kernel == 2 && tmem_supported(g) && tmem_fits(g, tmem_grid(g, n_layers)))
-      return launch_score_tmem(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
-                               v_layer_stride, vbar_in, scores, vbar_out, entropy,
-                               (char*)workspace, lay.off_tmem, (cudaStream_t)stream);
-    return launch_score_sm100(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
+      rc = launch_score_tmem(g, n_layers, q_win, k, v_used, q_layer_stride, k_layer_stride,
+                             v_layer_stride, vbar_in, scores, vbar_out, entropy,
+                             (char*)workspace, lay.off_tmem, st);
+    else
+      rc = launch_score_sm100(g, n_layers, q_win, k, v_used, q_layer_stride, k_layer_stride,
                               v_layer_stride, vbar_in, scores, vbar_out, entropy,
-                              (char*)workspace, lay.off_sm100, (cudaStream_t)stream);
+                              (char*)workspace, lay.off_sm100, st);
+  } else {
+    rc = launch_score_generic(g, n_layers, q_win, k, v_used, q_layer_stride, k_layer_stride,
+                              v_layer_stride, vbar_in, scores, vbar_out, entropy,
+                              (char*)workspace, lay, st);
   }
-  return launch_score_generic(g, n_layers, q_win, k, v, q_layer_stride, k_layer_stride,
-                              v_layer_stride, vbar_in, scores, vbar_out, entropy,
-                              (char*)workspace, lay, (cudaStream_t)stream);
+  if (rc != LAVA_OK || !token_term) return rc;
+  // VATP: every position's own value-row norm, then the entropy of the final scores
+  rc = launch_token_norm_scale(g, n_layers, v, v_layer_stride, scores, st);
+  if (rc != LAVA_OK) return rc;
+  return launch_entropy_from_scores(g, n_layers, scores, entropy, st);
 }
 
 lava_status lava_score_layer(const lava_layer_desc* desc, const void* q_win, const void* k,
@@ -302,7 +330,8 @@ lava_status lava_layer_budgets(int32_t n_layers, int32_t batch, const double* en
   if (!entropy || !total_budget || !floor_per_layer || !cap_per_layer || !layer_budget ||
       !layer_row_offset)
     return fail(LAVA_ERR_INVALID_ARG, "NULL argument");
-  if (mode != LAVA_BUDGET_DYNAMIC && mode != LAVA_BUDGET_UNIFORM)
+  if (mode < 0 || (mode & 0xff) > LAVA_BUDGET_PYRAMID || (mode >> 8) > 1000 ||
+      ((mode >> 8) != 0 && (mode & 0xff) != LAVA_BUDGET_PYRAMID))
     return fail(LAVA_ERR_INVALID_ARG, "unknown budget mode %d", mode);
   return launch_budgets(n_layers, batch, entropy, (const long long*)total_budget,
                         (const long long*)floor_per_layer, (const long long*)cap_per_layer, mode,

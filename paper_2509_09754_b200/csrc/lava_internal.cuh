@@ -13,7 +13,7 @@ namespace lava {
 // Geometry handed to kernels by value.
 struct Geom {
   int n_q_heads, n_kv_heads, group, head_dim, window, w_pad;
-  int pool_kind, pool_kernel, pool_radius, dtype, batch, max_seqlen;
+  int pool_kind, pool_kernel, pool_radius, dtype, batch, max_seqlen, flags;
   const int* cu_seqlens;
   long long total_tokens, total_scores;
   long long k_sh, k_st, v_sh, v_st;  // strides in elements
@@ -49,7 +49,7 @@ struct Workspace {
   static constexpr size_t kStatusBytes = 256;
   static constexpr int kSlice = 512;    // keys per block in the generic score kernels
   static constexpr int kVSlice = 1024;  // V rows per block in the value-norm kernel
-  size_t off_vpart, off_stats, off_lse, off_vbar, off_ent, off_sm100, off_tmem, total;
+  size_t off_vpart, off_stats, off_lse, off_vbar, off_ones, off_ent, off_sm100, off_tmem, total;
   int n_slices, n_vslices;
 };
 Workspace workspace_layout(const lava_layer_desc* d, int n_layers);
@@ -111,6 +111,12 @@ lava_status launch_score_tmem(const Geom& g, int n_layers, const void* q, const 
                               const void* v, long long q_ls, long long k_ls, long long v_ls,
                               const float* vbar_in, float* scores, float* vbar_out,
                               double* entropy, char* ws_base, size_t ws_off, cudaStream_t stream);
+lava_status launch_fill_ones(float* dst, long long count, cudaStream_t stream);
+lava_status launch_token_norm_scale(const Geom& g, int n_layers, const void* v, long long v_ls,
+                                    float* scores, cudaStream_t stream);
+// entropy of every (layer, sequence) from the final score array (fixed summation order)
+lava_status launch_entropy_from_scores(const Geom& g, int n_layers, const float* scores,
+                                       double* entropy, cudaStream_t stream);
 lava_status launch_wo_norm(const void* w_o, int dtype, long long rows, long long cols,
                            float* out, cudaStream_t stream);
 lava_status launch_budgets(int n_layers, int batch, const double* entropy,

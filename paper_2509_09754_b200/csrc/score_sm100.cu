@@ -1070,6 +1070,14 @@ int lead_extra_for(int chunk_tiles) {
 
 }  // namespace
 
+lava_status launch_entropy_from_scores(const Geom& g, int n_layers, const float* scores,
+                                       double* entropy, cudaStream_t stream) {
+  entropy_from_scores_kernel<<<n_layers * g.batch, 1024, 0, stream>>>(g, scores, entropy, nullptr,
+                                                                      nullptr, nullptr);
+  count_launches(1);
+  return check_cuda(cudaGetLastError(), "entropy launch");
+}
+
 bool sm100_supported(const Geom& g) {
   if (g.dtype != LAVA_BF16 || g.head_dim != 128) return false;
   if (g.window != 16 && g.window != 32 && g.window != 64 && g.window != 128) return false;

@@ -236,19 +236,33 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
   __shared__ RegShared sh;
   cg::cluster_group cluster = cg::this_cluster();
   const int csize = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
-  const int prob = blockIdx.x / csize, layer = prob / g.batch, b = prob - layer * g.batch;
+  // one cluster per (layer, sequence); with per-head selection (the "- head dynamic" ablation of
+  // Sec. 5.4) one per (layer, sequence, KV head), each on its head's segment alone
+  const bool per_head = (g.flags & LAVA_FLAG_PER_HEAD_TOPK) != 0;
+  const int cl = blockIdx.x / csize;
+  const int prob = per_head ? cl / g.n_kv_heads : cl, layer = prob / g.batch, b = prob - layer * g.batch;
+  const int head0 = per_head ? cl - prob * g.n_kv_heads : 0;  // first head of this problem
   const int lane = threadIdx.x & 31;
   const SeqInfo s = seq_info(g, b);
-  const int m_total = g.n_kv_heads * s.prefix;  // candidates (fits 31 bits)
-  const unsigned* keys =
-      reinterpret_cast<const unsigned*>(scores + (size_t)layer * g.total_scores + s.score_off);
-  int* out = keep_idx + (size_t)layer * g.total_scores + s.score_off;
-  int* hoff = head_offsets + (size_t)prob * (g.n_kv_heads + 1);
-
-  const long long window_rows = (long long)g.n_kv_heads * min(g.window, s.n);
+  const int m_total = (per_head ? 1 : g.n_kv_heads) * s.prefix;  // candidates (fits 31 bits)
+  const int win = min(g.window, s.n);
+  const long long window_rows = (long long)g.n_kv_heads * win;
   long long k_sel = layer_budget[prob] - window_rows;
   if (k_sel < 0) k_sel = 0;
+  int out_base = 0;  // kept entries of the heads before this problem's first head
+  if (per_head) {
+    // even shares of the selectable entries, the first (k mod H_kv) heads one more; a head
+    // never keeps more than it has
+    const long long share = k_sel / g.n_kv_heads, extra = k_sel % g.n_kv_heads;
+    out_base = share >= s.prefix ? head0 * s.prefix
+                                 : (int)(head0 * share + min((long long)head0, extra));
+    k_sel = share + (head0 < extra ? 1 : 0);
+  }
   if (k_sel > m_total) k_sel = m_total;
+  const unsigned* keys = reinterpret_cast<const unsigned*>(
+      scores + (size_t)layer * g.total_scores + s.score_off + (long long)head0 * s.prefix);
+  int* out = keep_idx + (size_t)layer * g.total_scores + s.score_off + out_base;
+  int* hoff = head_offsets + (size_t)prob * (g.n_kv_heads + 1);
 
   // this CTA's range; thread t owns its elements [t E, t E + E)
   const int per = (m_total + csize - 1) / csize;
@@ -397,9 +411,9 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
       const int pos0 = first - head * s.prefix;
       // heads that start inside this thread's keys record how many kept entries precede them
       for (int j = pos0 == 0 ? 0 : s.prefix - pos0; j < n_mine; j += s.prefix) {
-        const int h = (first + j) / s.prefix;
-        hoff[h] = (int)(kept_cta_before + slot0) + __popcll(keep_mask & ((1ull << j) - 1ull)) +
-                  h * g.window;
+        const int h = head0 + (first + j) / s.prefix;
+        hoff[h] = out_base + (int)(kept_cta_before + slot0) +
+                  __popcll(keep_mask & ((1ull << j) - 1ull)) + h * g.window;
       }
 #pragma unroll
       for (int j = 0; j < E; ++j) {
@@ -413,9 +427,14 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
     for (unsigned i = threadIdx.x; i < cta_kept; i += kThreads) out[kept_cta_before + i] = packed[i];
   }
   if (rank == 0 && threadIdx.x == 0) {
-    hoff[g.n_kv_heads] = (int)(k_sel + window_rows);
-    if (s.prefix == 0)  // no candidates: every head holds only its (possibly short) window
-      for (int h = 0; h < g.n_kv_heads; ++h) hoff[h] = h * min(g.window, s.n);
+    if (!per_head) {
+      hoff[g.n_kv_heads] = (int)(k_sel + window_rows);
+      if (s.prefix == 0)  // no candidates: every head holds only its (possibly short) window
+        for (int h = 0; h < g.n_kv_heads; ++h) hoff[h] = h * win;
+    } else {
+      if (s.prefix == 0) hoff[head0] = head0 * win;
+      if (head0 == g.n_kv_heads - 1) hoff[g.n_kv_heads] = out_base + (int)k_sel + (int)window_rows;
+    }
   }
   cluster.sync();  // peers may still be reading this CTA's counts
 }
@@ -455,9 +474,11 @@ lava_status launch_select(const Geom& g, int n_layers, const float* scores,
                           const long long* layer_budget, int* keep_idx, int* head_offsets,
                           unsigned* status, cudaStream_t stream) {
   (void)status;
+  const bool per_head = (g.flags & LAVA_FLAG_PER_HEAD_TOPK) != 0;
   // candidates of the largest problem; the register-resident kernel takes up to 32768 per CTA
-  const long long m_max = (long long)g.n_kv_heads * (g.max_seqlen > g.window ? g.max_seqlen - g.window : 0);
-  const int problems = n_layers * g.batch;
+  const long long m_max = (long long)(per_head ? 1 : g.n_kv_heads) *
+                          (g.max_seqlen > g.window ? g.max_seqlen - g.window : 0);
+  const int problems = n_layers * g.batch * (per_head ? g.n_kv_heads : 1);
   // 16 CTAs once a cluster of 8 would need 64 keys per thread: at 32 keys per thread two CTAs
   // share an SM
   int csize = m_max <= 8LL * (kRegMaxPerCta / 2) ? 8 : 16;
@@ -474,6 +495,8 @@ lava_status launch_select(const Geom& g, int n_layers, const float* scores,
     count_launches(1);
     return check_cuda(err, "select_topk launch");
   }
+  if (per_head)
+    return fail(LAVA_ERR_UNSUPPORTED, "per-head selection covers up to 524288 positions per head");
   dim3 grid(kCluster, n_layers * g.batch);
   select_topk_kernel<<<grid, kThreads, 0, stream>>>(g, scores, layer_budget, keep_idx,
                                                     head_offsets);
