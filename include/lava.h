@@ -267,6 +267,66 @@ LAVA_API lava_status lava_evict_model_host(const lava_layer_desc* desc, int32_t 
                                            int32_t* head_offsets, void* k_out, void* v_out,
                                            void* arena, size_t arena_bytes, void* stream);
 
+/* Layer-by-layer form of the method (Algorithm 2 and the paragraph after it): prefill and evict
+ * one layer at a time, so that only one layer's full K/V is ever alive.  After layer l has been
+ * scored, the budgets of layers 0..l are recomputed from e_0..e_l out of the total in force
+ * (the model's total, held inside [(l+1)*floor, (l+1)*cap] while few layers are live), layer l
+ * is evicted from its full K/V, and every lower layer is evicted again from what it still holds
+ * with the scores stored at its first eviction; only the retained scores are stored.  A second
+ * eviction can only drop entries, so the final cache equals the one-shot result of
+ * lava_layer_budgets / lava_select_topk / lava_compact_kv whenever no layer's budget ever grows
+ * from one step to the next.
+ *
+ *   lava_cascade_state_bytes  bytes of DEVICE memory the caller must provide as `state` for
+ *                     n_layers layers and an arena of total_rows packed rows (>= the sum of the
+ *                     sequences' total budgets).  Holds the packed K and V rows twice (each step
+ *                     writes the shrunken layout into the other copy), the held scores and
+ *                     positions twice, and one layer's full score and index arrays.
+ *   lava_cascade_create   validates and makes the HOST-side handle (owned by the caller, freed
+ *                     with lava_cascade_destroy; it owns no device memory).  `desc` is copied;
+ *                     desc->cu_seqlens and `state` must stay valid while the handle is used.
+ *                     mode is LAVA_BUDGET_DYNAMIC or LAVA_BUDGET_UNIFORM; LAVA_FLAG_PER_HEAD_TOPK
+ *                     is not supported here.  At most 524288 candidates per (layer, sequence).
+ *   lava_cascade_begin    total_budget: DEVICE int64 [batch], the model-wide budgets in rows.
+ *                     A total outside [L*floor, L*cap], or totals that exceed total_rows, are
+ *                     replaced by feasible ones and LAVA_DEV_BUDGET_INFEASIBLE is set in the
+ *                     status word of `workspace`.  Restarts the handle at layer 0.
+ *   lava_cascade_step     takes the next layer: q_win, k, v (and optional vbar_in) exactly as
+ *                     lava_score_layer, workspace of lava_workspace_bytes(desc, 1) bytes.  K and V
+ *                     of this layer may be released once the work enqueued here has finished.
+ *                     A step that returns an error leaves the handle unusable until the next
+ *                     lava_cascade_begin.
+ *   lava_cascade_get      device pointers into `state` for the layers taken so far (valid until
+ *                     the next step): rows and list entries of (layer l, sequence b) start at
+ *                     layer_row_offset[l*batch + b]; inside, head g's rows start at
+ *                     head_offsets[l][b][g] (kept prefix rows in ascending position, then the w
+ *                     window rows) and its kept positions / scores are list entries
+ *                     head_offsets[l][b][g] - g*w ... of that segment. */
+typedef struct lava_cascade lava_cascade;
+typedef struct lava_cascade_view {
+  int32_t layers_done;
+  void* k_out;                     /* packed rows [total_rows, d]                               */
+  void* v_out;
+  const int32_t* kept_pos;         /* [total_rows] positions of the kept prefix entries          */
+  const float* kept_scores;        /* [total_rows] their scores                                  */
+  const int32_t* head_offsets;     /* [layers_done, batch, H_kv+1]                               */
+  const int64_t* layer_budget;     /* [layers_done, batch]                                       */
+  const int64_t* layer_row_offset; /* [layers_done*batch + 1]                                    */
+  const double* entropy;           /* [layers_done, batch]                                       */
+} lava_cascade_view;
+LAVA_API size_t lava_cascade_state_bytes(const lava_layer_desc* desc, int32_t n_layers,
+                                         int64_t total_rows);
+LAVA_API lava_status lava_cascade_create(const lava_layer_desc* desc, int32_t n_layers,
+                                         int64_t total_rows, int32_t mode, void* state,
+                                         size_t state_bytes, lava_cascade** out);
+LAVA_API void lava_cascade_destroy(lava_cascade* h);
+LAVA_API lava_status lava_cascade_begin(lava_cascade* h, const int64_t* total_budget,
+                                        void* workspace, void* stream);
+LAVA_API lava_status lava_cascade_step(lava_cascade* h, const void* q_win, const void* k,
+                                       const void* v, const float* vbar_in, void* workspace,
+                                       size_t workspace_bytes, void* stream);
+LAVA_API lava_status lava_cascade_get(const lava_cascade* h, lava_cascade_view* out);
+
 /* Tuning and test knobs (no counterpart in the paper).  Process-wide; the defaults come from the
  * environment variables named below, read once when the library first needs an option, so no
  * call on the hot path reads the environment.  Set them while no call of this library is running.

@@ -390,8 +390,10 @@ def evict_model(q_win, k, v, w, total_budget, pool_kind=POOL_MAX, pool_kernel=7,
 # --------------------------------------------------------------------------------------------
 # Algorithm 2, streaming form: after each new layer, re-budget layers 0..l and re-evict them
 # --------------------------------------------------------------------------------------------
-def cascade_evict(scores, n, w, total_budget, mode=BUDGET_DYNAMIC):
-    """Follow Algorithm 2 on stored scores.  scores: list of [H_kv, P] arrays.
+def cascade_evict(scores, n, w, total_budget, mode=BUDGET_DYNAMIC, entropy=None):
+    """Follow Algorithm 2 on stored scores.  scores: list of [H_kv, P] arrays.  ``entropy``
+    (optional, [L]) supplies the e_l instead of layer_entropy(s_l): Algorithm 2 takes them as
+    given once computed, and a caller that compares integer budgets fixes them this way.
 
     After layer l arrives the budgets of layers 0..l are recomputed from e_0..e_l (the sum in
     the denominator runs over the layers prefilled so far) and every one of them is evicted
@@ -407,7 +409,7 @@ def cascade_evict(scores, n, w, total_budget, mode=BUDGET_DYNAMIC):
     monotone = True
     budgets = []
     for l, s in enumerate(scores):
-        ent.append(layer_entropy(s, n))
+        ent.append(layer_entropy(s, n) if entropy is None else float(entropy[l]))
         held.append(np.arange(n_kv_heads * prefix, dtype=np.int64))
         last_budget.append(hi)
         live = l + 1

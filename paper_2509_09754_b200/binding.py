@@ -37,6 +37,15 @@ class _CDesc(ctypes.Structure):
     ]
 
 
+class _CCascadeView(ctypes.Structure):
+    _fields_ = [
+        ("layers_done", ctypes.c_int32), ("k_out", ctypes.c_void_p), ("v_out", ctypes.c_void_p),
+        ("kept_pos", ctypes.c_void_p), ("kept_scores", ctypes.c_void_p),
+        ("head_offsets", ctypes.c_void_p), ("layer_budget", ctypes.c_void_p),
+        ("layer_row_offset", ctypes.c_void_p), ("entropy", ctypes.c_void_p),
+    ]
+
+
 _LIB = None
 
 
@@ -84,6 +93,16 @@ def load_library():
     lib.lava_set_option.argtypes = [ctypes.c_char_p, i64]
     lib.lava_get_option.restype = i64
     lib.lava_get_option.argtypes = [ctypes.c_char_p]
+    lib.lava_cascade_state_bytes.restype = sz
+    lib.lava_cascade_state_bytes.argtypes = [dp, i32, i64]
+    lib.lava_cascade_create.argtypes = [dp, i32, i64, i32, vp, sz, ctypes.POINTER(vp)]
+    lib.lava_cascade_destroy.restype = None
+    lib.lava_cascade_destroy.argtypes = [vp]
+    lib.lava_cascade_begin.argtypes = [vp, vp, vp, vp]
+    lib.lava_cascade_step.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_cascade_get.argtypes = [vp, ctypes.POINTER(_CCascadeView)]
+    for name in ("lava_cascade_create", "lava_cascade_begin", "lava_cascade_step", "lava_cascade_get"):
+        getattr(lib, name).restype = i32
     for name in ("lava_poll_status", "lava_wo_norm", "lava_score_layer", "lava_score_layers",
                  "lava_layer_budgets", "lava_select_topk", "lava_select_topk_layers",
                  "lava_compact_kv", "lava_compact_kv_layers"):
@@ -338,6 +357,75 @@ def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC
     lava_compact_kv_layers(d, nl, k, v, k.stride(0), v.stride(0), plan.keep_idx,
                            plan.head_offsets, plan.layer_row_offset, plan.k_out, plan.v_out,
                            stream)
+
+
+# ----------------------------------------------------------------------------- layer by layer
+def lava_cascade_state_bytes(desc: LayerDesc, n_layers: int, total_rows: int) -> int:
+    n = load_library().lava_cascade_state_bytes(ctypes.byref(desc.to_c()), n_layers, int(total_rows))
+    if n == 0:
+        raise LavaError(1, "invalid layer descriptor, layer count or row count")
+    return n
+
+
+class Cascade:
+    """Algorithm 2, one layer per call (lava_cascade_* of the C ABI).  Owns the device state block
+    and a one-layer workspace; `step` takes the layers in order, `view` returns tensors that alias
+    the state (valid until the next step)."""
+
+    def __init__(self, desc: LayerDesc, n_layers: int, total_rows: int,
+                 mode: int = LAVA_BUDGET_DYNAMIC, device="cuda", kv_dtype=torch.bfloat16):
+        self.desc, self.n_layers, self.total_rows, self.kv_dtype = desc, n_layers, int(total_rows), kv_dtype
+        self._cdesc = desc.to_c()
+        self.state = torch.zeros(lava_cascade_state_bytes(desc, n_layers, total_rows),
+                                 dtype=torch.uint8, device=device)
+        self.workspace = torch.zeros(lava_workspace_bytes(desc, 1), dtype=torch.uint8, device=device)
+        self._h = ctypes.c_void_p()
+        _check(load_library().lava_cascade_create(
+            ctypes.byref(self._cdesc), n_layers, self.total_rows, mode, _ptr(self.state),
+            self.state.numel(), ctypes.byref(self._h)))
+
+    def close(self):
+        if self._h:
+            load_library().lava_cascade_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def begin(self, total_budget: torch.Tensor, stream=None) -> None:
+        _check(load_library().lava_cascade_begin(self._h, _ptr(total_budget), _ptr(self.workspace),
+                                                 _stream(stream)))
+
+    def step(self, q_win, k, v, vbar_in=None, stream=None) -> None:
+        _check(load_library().lava_cascade_step(self._h, _ptr(q_win), _ptr(k), _ptr(v), _ptr(vbar_in),
+                                                _ptr(self.workspace), self.workspace.numel(),
+                                                _stream(stream)))
+
+    def view(self) -> dict:
+        cv = _CCascadeView()
+        _check(load_library().lava_cascade_get(self._h, ctypes.byref(cv)))
+        d, done, base = self.desc, cv.layers_done, self.state.data_ptr()
+
+        def at(ptr, nbytes, dtype, shape):
+            off = ptr - base
+            return self.state[off: off + nbytes].view(dtype).view(shape)
+
+        es = 2 if self.kv_dtype == torch.bfloat16 else 4
+        rows, lb = self.total_rows, done * d.batch
+        return dict(
+            layers_done=done,
+            k_out=at(cv.k_out, rows * d.head_dim * es, self.kv_dtype, (rows, d.head_dim)),
+            v_out=at(cv.v_out, rows * d.head_dim * es, self.kv_dtype, (rows, d.head_dim)),
+            kept_pos=at(cv.kept_pos, rows * 4, torch.int32, (rows,)),
+            kept_scores=at(cv.kept_scores, rows * 4, torch.float32, (rows,)),
+            head_offsets=at(cv.head_offsets, lb * (d.n_kv_heads + 1) * 4, torch.int32,
+                            (done, d.batch, d.n_kv_heads + 1)),
+            layer_budget=at(cv.layer_budget, lb * 8, torch.int64, (done, d.batch)),
+            layer_row_offset=at(cv.layer_row_offset, (lb + 1) * 8, torch.int64, (lb + 1,)),
+            entropy=at(cv.entropy, lb * 8, torch.float64, (done, d.batch)))
 
 
 # ----------------------------------------------------------------------------- host buffers

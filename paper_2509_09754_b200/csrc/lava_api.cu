@@ -62,7 +62,6 @@ int sm_count() {
   return n;
 }
 
-static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -67,6 +67,8 @@ struct Options {
 Options& options();
 int sm_count();            // multiprocessors of the current device (cached per device), 0 on error
 
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
 // Host-side error plumbing.
 lava_status fail(lava_status st, const char* fmt, ...);
 lava_status check_cuda(cudaError_t e, const char* what);
@@ -126,6 +128,24 @@ lava_status launch_budgets(int n_layers, int batch, const double* entropy,
 lava_status launch_select(const Geom& g, int n_layers, const float* scores,
                           const long long* layer_budget, int* keep_idx, int* head_offsets,
                           unsigned* status, cudaStream_t stream);
+// Lists of what every (layer, sequence) still holds during Algorithm 2's cascade: score and
+// position of each held prefix entry, heads in order and positions ascending inside a head; the
+// list of problem p starts at entry row_off[p] and its heads are delimited like the packed rows
+// (head g's entries start at head_offsets[p][g] - g*w).
+struct HeldLists {
+  const float* score_old = nullptr;
+  const int* pos_old = nullptr;
+  const long long* row_off_old = nullptr;
+  const int* hoff_old = nullptr;
+  float* score_new = nullptr;
+  int* pos_new = nullptr;
+  int* src_pos = nullptr;           // for every new entry: its index in the old list
+  const long long* row_off_new = nullptr;
+};
+// Re-selection of `problems` (layer, sequence) lists, each down to layer_budget[p] rows.
+lava_status launch_reselect(const Geom& g, int problems, long long max_held,
+                            const long long* layer_budget, int* head_offsets_new,
+                            const HeldLists& io, cudaStream_t stream);
 lava_status launch_compact(const Geom& g, int n_layers, const void* k, const void* v,
                            long long k_ls, long long v_ls, const int* keep_idx,
                            const int* head_offsets, const long long* row_off, void* k_out,

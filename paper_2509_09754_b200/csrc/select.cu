@@ -227,10 +227,15 @@ struct RegCfg {
   static constexpr int kBigWords = kStageWords > kHistWords ? kStageWords : kHistWords;
 };
 
-template <int E>
+// LIST selects among the entries a layer still holds (Algorithm 2: a lower layer is evicted
+// again with its stored scores): the keys of problem p are the `held` scores of its list, in
+// list order, which is ascending flat index, so ties still go to the lower flat index.  The
+// kept entries' scores and positions are copied to the new list and `src_pos` records where in
+// the old list each came from.
+template <int E, bool LIST>
 __global__ void __launch_bounds__(kThreads, RegCfg<E>::kMinCtas)
 select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budget, int* keep_idx,
-                       int* head_offsets) {
+                       int* head_offsets, HeldLists io) {
   using Cfg = RegCfg<E>;
   extern __shared__ __align__(16) unsigned big[];  // staging / histogram copies / packed output
   __shared__ RegShared sh;
@@ -238,14 +243,17 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
   const int csize = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   // one cluster per (layer, sequence); with per-head selection (the "- head dynamic" ablation of
   // Sec. 5.4) one per (layer, sequence, KV head), each on its head's segment alone
-  const bool per_head = (g.flags & LAVA_FLAG_PER_HEAD_TOPK) != 0;
+  const bool per_head = !LIST && (g.flags & LAVA_FLAG_PER_HEAD_TOPK) != 0;
   const int cl = blockIdx.x / csize;
   const int prob = per_head ? cl / g.n_kv_heads : cl, layer = prob / g.batch, b = prob - layer * g.batch;
   const int head0 = per_head ? cl - prob * g.n_kv_heads : 0;  // first head of this problem
   const int lane = threadIdx.x & 31;
   const SeqInfo s = seq_info(g, b);
-  const int m_total = (per_head ? 1 : g.n_kv_heads) * s.prefix;  // candidates (fits 31 bits)
   const int win = min(g.window, s.n);
+  const int* hoff_old = LIST ? io.hoff_old + (size_t)prob * (g.n_kv_heads + 1) : nullptr;
+  // candidates (fits 31 bits): the whole prefix of every head, or what the list still holds
+  const int m_total = LIST ? max(0, hoff_old[g.n_kv_heads] - g.n_kv_heads * win)
+                           : (per_head ? 1 : g.n_kv_heads) * s.prefix;
   const long long window_rows = (long long)g.n_kv_heads * win;
   long long k_sel = layer_budget[prob] - window_rows;
   if (k_sel < 0) k_sel = 0;
@@ -259,9 +267,12 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
     k_sel = share + (head0 < extra ? 1 : 0);
   }
   if (k_sel > m_total) k_sel = m_total;
+  const long long old0 = LIST ? io.row_off_old[prob] : 0, new0 = LIST ? io.row_off_new[prob] : 0;
   const unsigned* keys = reinterpret_cast<const unsigned*>(
-      scores + (size_t)layer * g.total_scores + s.score_off + (long long)head0 * s.prefix);
-  int* out = keep_idx + (size_t)layer * g.total_scores + s.score_off + out_base;
+      LIST ? io.score_old + old0
+           : scores + (size_t)layer * g.total_scores + s.score_off + (long long)head0 * s.prefix);
+  int* out = LIST ? io.pos_new + new0
+                  : keep_idx + (size_t)layer * g.total_scores + s.score_off + out_base;
   int* hoff = head_offsets + (size_t)prob * (g.n_kv_heads + 1);
 
   // this CTA's range; thread t owns its elements [t E, t E + E)
@@ -405,6 +416,30 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
       }
     }
     int* packed = reinterpret_cast<int*>(big);
+    if (LIST) {
+      if (n_mine > 0) {
+        const int first = c0 + (int)threadIdx.x * E;
+        // heads whose list segment starts inside this thread's keys
+        for (int h = 0; h < g.n_kv_heads; ++h) {
+          const int j = hoff_old[h] - h * win - first;
+          if (j >= 0 && j < n_mine)
+            hoff[h] = (int)(kept_cta_before + slot0) + __popcll(keep_mask & ((1ull << j) - 1ull)) +
+                      h * win;
+        }
+#pragma unroll
+        for (int j = 0; j < E; ++j)
+          if ((keep_mask >> j) & 1ull)
+            packed[slot0 + __popcll(keep_mask & ((1ull << j) - 1ull))] = first + j;
+      }
+      __syncthreads();
+      for (unsigned i = threadIdx.x; i < cta_kept; i += kThreads) {
+        const int p = packed[i];
+        const long long o = new0 + kept_cta_before + i;
+        io.pos_new[o] = io.pos_old[old0 + p];
+        io.score_new[o] = io.score_old[old0 + p];
+        io.src_pos[o] = p;
+      }
+    } else {
     if (n_mine > 0) {
       const int first = c0 + (int)threadIdx.x * E;
       int head = first / s.prefix;
@@ -425,9 +460,15 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
     }
     __syncthreads();
     for (unsigned i = threadIdx.x; i < cta_kept; i += kThreads) out[kept_cta_before + i] = packed[i];
+    }
   }
   if (rank == 0 && threadIdx.x == 0) {
-    if (!per_head) {
+    if (LIST) {
+      // heads whose segment starts past the last held entry (empty tail heads, or an empty list)
+      for (int h = 0; h < g.n_kv_heads; ++h)
+        if (hoff_old[h] - h * win >= m_total) hoff[h] = (int)k_sel + h * win;
+      hoff[g.n_kv_heads] = (int)k_sel + g.n_kv_heads * win;
+    } else if (!per_head) {
       hoff[g.n_kv_heads] = (int)(k_sel + window_rows);
       if (s.prefix == 0)  // no candidates: every head holds only its (possibly short) window
         for (int h = 0; h < g.n_kv_heads; ++h) hoff[h] = h * win;
@@ -439,11 +480,11 @@ select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budge
   cluster.sync();  // peers may still be reading this CTA's counts
 }
 
-template <int E>
+template <int E, bool LIST = false>
 cudaError_t launch_reg(const Geom& g, int problems, int csize, const float* scores,
                        const long long* layer_budget, int* keep_idx, int* head_offsets,
-                       cudaStream_t stream) {
-  auto kern = select_topk_reg_kernel<E>;
+                       cudaStream_t stream, HeldLists io = HeldLists()) {
+  auto kern = select_topk_reg_kernel<E, LIST>;
   const int big_bytes = RegCfg<E>::kBigWords * (int)sizeof(unsigned);
   {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, big_bytes);
@@ -465,7 +506,7 @@ cudaError_t launch_reg(const Geom& g, int problems, int csize, const float* scor
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, g, scores, layer_budget, keep_idx, head_offsets);
+  return cudaLaunchKernelEx(&cfg, kern, g, scores, layer_budget, keep_idx, head_offsets, io);
 }
 
 }  // namespace
@@ -502,6 +543,25 @@ lava_status launch_select(const Geom& g, int n_layers, const float* scores,
                                                     head_offsets);
   count_launches(1);
   return check_cuda(cudaGetLastError(), "select_topk launch");
+}
+
+lava_status launch_reselect(const Geom& g, int problems, long long max_held,
+                            const long long* layer_budget, int* head_offsets_new,
+                            const HeldLists& io, cudaStream_t stream) {
+  if (problems < 1) return LAVA_OK;
+  int csize = max_held <= 8LL * (kRegMaxPerCta / 2) ? 8 : 16;
+  if (max_held > (long long)csize * kRegMaxPerCta)
+    return fail(LAVA_ERR_UNSUPPORTED, "a layer may hold at most %d entries per sequence here",
+                16 * kRegMaxPerCta);
+  const long long per = (max_held + csize - 1) / csize;
+  const int e = (int)((per + kThreads - 1) / kThreads);
+  cudaError_t err;
+  if (e <= 8) err = launch_reg<8, true>(g, problems, csize, nullptr, layer_budget, nullptr, head_offsets_new, stream, io);
+  else if (e <= 16) err = launch_reg<16, true>(g, problems, csize, nullptr, layer_budget, nullptr, head_offsets_new, stream, io);
+  else if (e <= 32) err = launch_reg<32, true>(g, problems, csize, nullptr, layer_budget, nullptr, head_offsets_new, stream, io);
+  else err = launch_reg<64, true>(g, problems, csize, nullptr, layer_budget, nullptr, head_offsets_new, stream, io);
+  count_launches(1);
+  return check_cuda(err, "reselect launch");
 }
 
 }  // namespace lava
