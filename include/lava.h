@@ -327,6 +327,28 @@ LAVA_API lava_status lava_cascade_step(lava_cascade* h, const void* q_win, const
                                        size_t workspace_bytes, void* stream);
 LAVA_API lava_status lava_cascade_get(const lava_cascade* h, lava_cascade_view* out);
 
+/* Evaluator (not on the eviction path): layer attention output loss of a selection, Lemma 1 with
+ * p = 1 for the last token of every sequence, and the upper bound of Theorem 1:
+ *     loss[b]  = || Cat_h[ (A_h - A^_h) V_g(h) ] W_O ||_1 ,  A^_h = (A_h (.) I) / ||A_h (.) I||_1
+ *     bound[b] = 2 ||W_O^T||_1 sum_h Vbar_g(h) sum_i A_h[i] (1 - I_g(h)[i])
+ * where A_h is the softmax attention row of the last token over all keys of its sequence and I
+ * marks the retained entries of KV head g(h) (kept prefix positions and the window).
+ *   q_win, k, v        one layer, as in lava_score_layer (the last row of the window is the query)
+ *   keep_idx, head_offsets   the layer's selection, as written by lava_select_topk
+ *   vbar               [batch, H_kv] value norms of the layer (vbar_out of lava_score_layer)
+ *   w_o                DEVICE row-major [H_q*d, d_model], dtype w_o_dtype (lava_dtype)
+ *   loss_out, bound_out   DEVICE double [batch]
+ *   workspace          at least lava_loss_workspace_bytes(desc, d_model) bytes (holds the attention
+ *                      rows as doubles: 8*H_q*total_tokens bytes, plus small arrays)
+ * Sums are taken in double in a fixed order. */
+LAVA_API size_t lava_loss_workspace_bytes(const lava_layer_desc* desc, int64_t d_model);
+LAVA_API lava_status lava_layer_output_loss(const lava_layer_desc* desc, const void* q_win,
+                                            const void* k, const void* v, const int32_t* keep_idx,
+                                            const int32_t* head_offsets, const float* vbar,
+                                            const void* w_o, int32_t w_o_dtype, int64_t d_model,
+                                            double* loss_out, double* bound_out, void* workspace,
+                                            size_t workspace_bytes, void* stream);
+
 /* Tuning and test knobs (no counterpart in the paper).  Process-wide; the defaults come from the
  * environment variables named below, read once when the library first needs an option, so no
  * call on the hot path reads the environment.  Set them while no call of this library is running.

@@ -93,6 +93,10 @@ def load_library():
     lib.lava_set_option.argtypes = [ctypes.c_char_p, i64]
     lib.lava_get_option.restype = i64
     lib.lava_get_option.argtypes = [ctypes.c_char_p]
+    lib.lava_loss_workspace_bytes.restype = sz
+    lib.lava_loss_workspace_bytes.argtypes = [dp, i64]
+    lib.lava_layer_output_loss.restype = i32
+    lib.lava_layer_output_loss.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lava_cascade_state_bytes.restype = sz
     lib.lava_cascade_state_bytes.argtypes = [dp, i32, i64]
     lib.lava_cascade_create.argtypes = [dp, i32, i64, i32, vp, sz, ctypes.POINTER(vp)]
@@ -357,6 +361,21 @@ def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC
     lava_compact_kv_layers(d, nl, k, v, k.stride(0), v.stride(0), plan.keep_idx,
                            plan.head_offsets, plan.layer_row_offset, plan.k_out, plan.v_out,
                            stream)
+
+
+def lava_layer_output_loss(desc: LayerDesc, q_win, k, v, keep_idx, head_offsets, vbar, w_o,
+                           loss_out, bound_out, workspace=None, stream=None):
+    """Lemma 1 loss (p = 1, last token) and Theorem 1 bound of one layer's selection."""
+    lib = load_library()
+    d_model = int(w_o.shape[1])
+    need = lib.lava_loss_workspace_bytes(ctypes.byref(desc.to_c()), d_model)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=k.device)
+    _check(lib.lava_layer_output_loss(
+        ctypes.byref(desc.to_c()), _ptr(q_win), _ptr(k), _ptr(v), _ptr(keep_idx), _ptr(head_offsets),
+        _ptr(vbar), _ptr(w_o), _dtype_code(w_o), d_model, _ptr(loss_out), _ptr(bound_out),
+        _ptr(workspace), workspace.numel(), _stream(stream)))
+    return workspace
 
 
 # ----------------------------------------------------------------------------- layer by layer
