@@ -327,6 +327,33 @@ LAVA_API lava_status lava_cascade_step(lava_cascade* h, const void* q_win, const
                                        size_t workspace_bytes, void* stream);
 LAVA_API lava_status lava_cascade_get(const lava_cascade* h, lava_cascade_view* out);
 
+/* Consumer of the packed cache: the attention of one new token per sequence over the retained
+ * rows (Sec. 2 attention restricted to K-hat, V-hat of Algorithm 1).  After the layer-wide
+ * selection every KV head holds its own number of rows; query head h reads KV head
+ * g = h / (H_q / H_kv):   out[h] = softmax_i(sm_scale * q[h] . K-hat_g[i]) V-hat_g.
+ *   q                 [n_layers, batch, H_q, d] queries of the new token, dtype desc->dtype
+ *   k_packed, v_packed   the packed caches written by lava_compact_kv (or a cascade's k_out, v_out)
+ *   head_offsets      [n_layers, batch, H_kv+1] as written by lava_select_topk
+ *   layer_row_offset  [n_layers*batch (+1)]
+ *   out               float [n_layers, batch, H_q, d]; a head without rows gives zeros
+ *   workspace         lava_decode_workspace_bytes(desc, n_layers) bytes (partial results of the
+ *                     warps that share a head; unused outside bf16 / d = 128 / group <= 8)
+ * bf16 with d = 128 runs on the tensor path with the probabilities rounded to bf16 before they
+ * multiply V (error <= 2^-8 * sum_i p_i |V[i][c]| per output); other geometries run a plain
+ * fp32 kernel.  lava_decode_attention is the one-layer form (pointers of that layer). */
+LAVA_API size_t lava_decode_workspace_bytes(const lava_layer_desc* desc, int32_t n_layers);
+LAVA_API lava_status lava_decode_attention_layers(const lava_layer_desc* desc, int32_t n_layers,
+                                                  const void* q, const void* k_packed,
+                                                  const void* v_packed, const int32_t* head_offsets,
+                                                  const int64_t* layer_row_offset, float* out,
+                                                  void* workspace, size_t workspace_bytes,
+                                                  void* stream);
+LAVA_API lava_status lava_decode_attention(const lava_layer_desc* desc, const void* q,
+                                           const void* k_packed, const void* v_packed,
+                                           const int32_t* head_offsets,
+                                           const int64_t* layer_row_offset, float* out,
+                                           void* workspace, size_t workspace_bytes, void* stream);
+
 /* Evaluator (not on the eviction path): layer attention output loss of a selection, Lemma 1 with
  * p = 1 for the last token of every sequence, and the upper bound of Theorem 1:
  *     loss[b]  = || Cat_h[ (A_h - A^_h) V_g(h) ] W_O ||_1 ,  A^_h = (A_h (.) I) / ||A_h (.) I||_1

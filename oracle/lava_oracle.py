@@ -435,6 +435,35 @@ def cascade_evict(scores, n, w, total_budget, mode=BUDGET_DYNAMIC, entropy=None)
 
 
 # --------------------------------------------------------------------------------------------
+# The consumer of the compressed cache: one decoding step's attention (Sec. 2 attention over
+# the retained entries K-hat, V-hat of Algorithm 1; each KV head keeps its own number of rows)
+# --------------------------------------------------------------------------------------------
+def decode_attention(q, k_rows, v_rows, sm_scale=None):
+    """out[h] = softmax_i(sm_scale * q[h] . K-hat_g[i]) V-hat_g, g = h // (H_q // H_kv).
+
+    q      : [H_q, d] the new token's query heads
+    k_rows : list over KV heads of [len_g, d] retained key rows (any order: a softmax-weighted
+             sum does not depend on it); v_rows likewise
+    returns [H_q, d] fp64; a head with no rows gives zeros.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    n_q_heads, d = q.shape
+    group = n_q_heads // len(k_rows)
+    scale = (1.0 / math.sqrt(d)) if sm_scale in (None, 0, 0.0) else float(sm_scale)
+    out = np.zeros((n_q_heads, d), dtype=np.float64)
+    for h in range(n_q_heads):
+        kk = np.asarray(k_rows[h // group], dtype=np.float64)
+        vv = np.asarray(v_rows[h // group], dtype=np.float64)
+        if kk.shape[0] == 0:
+            continue
+        z = scale * (kk @ q[h])
+        z = z - z.max()
+        e = np.exp(z)
+        out[h] = (e / e.sum()) @ vv
+    return out
+
+
+# --------------------------------------------------------------------------------------------
 # Lemma 1 and Theorem 1 evaluators (used only to pin the scoring rule on tiny inputs)
 # --------------------------------------------------------------------------------------------
 def masked_attention(att_row, mask):

@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     lava_version, lava_last_error, lava_workspace_bytes, lava_poll_status, lava_wo_norm,
     lava_score_layer, lava_score_layer_static, lava_score_layers, lava_layer_budgets,
     lava_select_topk, lava_select_topk_layers, lava_compact_kv, lava_compact_kv_layers,
-    EvictionPlan, evict_model, lava_layer_output_loss, Cascade, lava_cascade_state_bytes,
+    EvictionPlan, evict_model, lava_layer_output_loss,
+    lava_decode_workspace_bytes, lava_decode_attention_layers, lava_decode_attention, Cascade, lava_cascade_state_bytes,
     lava_launch_count, lava_score_path, lava_set_option, lava_get_option, lava_host_arena_bytes, lava_evict_model_host,
 )

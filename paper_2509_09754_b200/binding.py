@@ -93,6 +93,12 @@ def load_library():
     lib.lava_set_option.argtypes = [ctypes.c_char_p, i64]
     lib.lava_get_option.restype = i64
     lib.lava_get_option.argtypes = [ctypes.c_char_p]
+    lib.lava_decode_workspace_bytes.restype = sz
+    lib.lava_decode_workspace_bytes.argtypes = [dp, i32]
+    lib.lava_decode_attention_layers.restype = i32
+    lib.lava_decode_attention_layers.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.lava_decode_attention.restype = i32
+    lib.lava_decode_attention.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.lava_loss_workspace_bytes.restype = sz
     lib.lava_loss_workspace_bytes.argtypes = [dp, i64]
     lib.lava_layer_output_loss.restype = i32
@@ -361,6 +367,26 @@ def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC
     lava_compact_kv_layers(d, nl, k, v, k.stride(0), v.stride(0), plan.keep_idx,
                            plan.head_offsets, plan.layer_row_offset, plan.k_out, plan.v_out,
                            stream)
+
+
+def lava_decode_workspace_bytes(desc: LayerDesc, n_layers: int = 1) -> int:
+    return load_library().lava_decode_workspace_bytes(ctypes.byref(desc.to_c()), n_layers)
+
+
+def lava_decode_attention_layers(desc: LayerDesc, n_layers, q, k_packed, v_packed, head_offsets,
+                                 layer_row_offset, out, workspace, stream=None) -> None:
+    _check(load_library().lava_decode_attention_layers(
+        ctypes.byref(desc.to_c()), n_layers, _ptr(q), _ptr(k_packed), _ptr(v_packed),
+        _ptr(head_offsets), _ptr(layer_row_offset), _ptr(out), _ptr(workspace),
+        0 if workspace is None else workspace.numel(), _stream(stream)))
+
+
+def lava_decode_attention(desc: LayerDesc, q, k_packed, v_packed, head_offsets, layer_row_offset,
+                          out, workspace, stream=None) -> None:
+    _check(load_library().lava_decode_attention(
+        ctypes.byref(desc.to_c()), _ptr(q), _ptr(k_packed), _ptr(v_packed), _ptr(head_offsets),
+        _ptr(layer_row_offset), _ptr(out), _ptr(workspace),
+        0 if workspace is None else workspace.numel(), _stream(stream)))
 
 
 def lava_layer_output_loss(desc: LayerDesc, q_win, k, v, keep_idx, head_offsets, vbar, w_o,

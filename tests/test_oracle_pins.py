@@ -533,3 +533,51 @@ def test_value_term_variants():
     tok2[1, 7] = tok[1, 7]
     np.testing.assert_array_equal(tok2, tok)
     np.testing.assert_allclose(O.token_value_norms(v_one)[1, 7], 5.0 * d, rtol=1e-13)
+
+
+# ------------------------------------------------------------------ the consumer: decode attention
+def test_decode_attention_special_cases_and_library_softmax():
+    rng = np.random.RandomState(11)
+    d, hq, hkv = 8, 4, 2
+    q = rng.randn(hq, d)
+    # one retained row: the output is that row of V, whatever the logit
+    k1 = [rng.randn(1, d) for _ in range(hkv)]
+    v1 = [rng.randn(1, d) for _ in range(hkv)]
+    out = O.decode_attention(q, k1, v1)
+    for h in range(hq):
+        np.testing.assert_allclose(out[h], v1[h // 2][0], rtol=1e-13)
+    # identical keys: uniform weights, the plain mean of the value rows
+    kk = [np.tile(rng.randn(1, d), (5, 1)), np.tile(rng.randn(1, d), (3, 1))]
+    vv = [rng.randn(5, d), rng.randn(3, d)]
+    out = O.decode_attention(q, kk, vv)
+    for h in range(hq):
+        np.testing.assert_allclose(out[h], vv[h // 2].mean(axis=0), rtol=1e-12)
+    # a head with no rows gives zeros; lengths differ per head
+    out = O.decode_attention(q, [np.zeros((0, d)), kk[1]], [np.zeros((0, d)), vv[1]])
+    assert np.all(out[:2] == 0.0) and np.any(out[2:] != 0.0)
+    # against the library softmax, with an explicit scale (a transposed product, a missing scale
+    # or the wrong head grouping would show)
+    kr = [rng.randn(7, d), rng.randn(4, d)]
+    vr = [rng.randn(7, d), rng.randn(4, d)]
+    out = O.decode_attention(q, kr, vr, sm_scale=0.37)
+    for h in range(hq):
+        g = h // 2
+        p = torch.softmax(torch.tensor(0.37 * kr[g] @ q[h]), dim=0).numpy()
+        np.testing.assert_allclose(out[h], p @ vr[g], rtol=1e-12)
+    # row order does not matter
+    perm = rng.permutation(7)
+    out2 = O.decode_attention(q, [kr[0][perm], kr[1]], [vr[0][perm], vr[1]], sm_scale=0.37)
+    np.testing.assert_allclose(out2, out, rtol=1e-12)
+
+
+def test_decode_attention_over_a_full_cache_is_the_last_attention_row_times_v():
+    """Nothing evicted: the new token's output equals the (already pinned) attention row of a
+    query at the last position applied to V."""
+    rng = np.random.RandomState(12)
+    hq, hkv, n, d, w = 4, 2, 19, 8, 3
+    q_win = rng.randn(hq, w, d)
+    k, v = rng.randn(hkv, n, d), rng.randn(hkv, n, d)
+    att = O.window_attention(q_win, k)[:, w - 1, :]                      # sees all n keys
+    out = O.decode_attention(q_win[:, w - 1, :], list(k), list(v))
+    for h in range(hq):
+        np.testing.assert_allclose(out[h], att[h] @ v[h // 2], rtol=1e-12)
