@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--path", default="evict", choices=["evict", "cascade", "decode"],
+                    help="evict: the one-shot hot path (the headline line); cascade: Algorithm 2 one "
+                         "layer per call; decode: attention of one new token over the packed cache")
     ap.add_argument("--layers", type=int, default=0,
                     help="run only the first N layers of the workload (small cases for profiling; "
                          "the budget shrinks in proportion and the line says so)")
@@ -264,6 +267,83 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- further paths
+def run_next_path(args, cfg, plan, q, k, v, stream, steps, warmup, local_rank, rank, world):
+    """The layer-by-layer cascade (Algorithm 2) or the decode-time consumer of the packed cache,
+    timed like the headline path (CUDA events, clocks sampled, one JSON line)."""
+    import torch
+    import paper_2509_09754_b200 as lava
+    from paper_2509_09754_b200 import replicas
+
+    L, d = cfg.n_layers, cfg.head_dim
+    es = 2 if cfg.dtype == "bf16" else 4
+    rows = int(plan.total_budget.sum().item())
+    peak, peak_src = measured_hbm_peak()
+    kv_bytes, out_bytes = roofline_bytes(cfg)
+    if args.path == "cascade":
+        cas = lava.Cascade(plan.desc, L, rows, kv_dtype=q.dtype, device=q.device)
+
+        def step():
+            cas.begin(plan.total_budget, stream)
+            for l in range(L):
+                cas.step(q[l], k[l], v[l], stream=stream)
+        metric, unit, units = "context tokens/s per layer-by-layer eviction (Algorithm 2)", UNIT, cfg.total_tokens
+        alg_bytes = kv_bytes + out_bytes
+        note = ("K + V read once + the final packed cache; every step also re-evicts all lower "
+                "layers (rows moved once per step), which this figure does not credit")
+        workspace = cas.workspace
+    else:
+        dev = q.device
+        gen = torch.Generator(device="cpu").manual_seed(3)
+        q_new = torch.randn((L, cfg.batch, cfg.n_q_heads, d), generator=gen).to(q.dtype).to(dev)
+        out = torch.empty((L, cfg.batch, cfg.n_q_heads, d), dtype=torch.float32, device=dev)
+        ws = torch.empty(max(256, lava.lava_decode_workspace_bytes(plan.desc, L)), dtype=torch.uint8,
+                         device=dev)
+
+        def step():
+            lava.lava_decode_attention_layers(plan.desc, L, q_new, plan.k_out, plan.v_out,
+                                              plan.head_offsets, plan.layer_row_offset, out, ws, stream)
+        metric, unit, units = "cached KV rows/s read by one decode step over all layers", "rows/s", rows
+        alg_bytes = rows * 2 * d * es
+        note = "one K row and one V row per retained (KV head, position), read once for the whole query group"
+        workspace = plan.workspace
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    launches0 = lava.lava_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    sampler.start()
+    ev[0].record(stream)
+    for i in range(steps):
+        step()
+        ev[i + 1].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    status = lava.lava_poll_status(workspace)
+    if status != 0:
+        raise SystemExit("device status word %d" % status)
+    per_step = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
+    ms = replicas.slowest_rank_ms(ev[0].elapsed_time(ev[steps])) / steps
+    gbs = alg_bytes / (ms * 1e-3) / 1e9
+    if rank == 0:
+        print(json.dumps({
+            "metric": metric, "value": replicas.whole_job_units(units) / (ms * 1e-3), "unit": unit,
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms,
+            "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": per_step[0],
+            "ms_per_step_max": per_step[-1], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "path": args.path, "n_layers": L,
+                       "seq_lens": list(cfg.seq_lens), "packed_rows": rows,
+                       "l2": "the packed cache and the inputs exceed the 126 MB L2; no flush"
+                             if alg_bytes > 126e6 else "working set below L2: not an HBM number"},
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                         "frac": gbs / peak, "traffic": None, "peak_source": peak_src,
+                         "algorithmic_bytes": alg_bytes, "note": note},
+            "e2e": None, "cpu_baseline": None,
+            "gpu_launches": lava.lava_launch_count() - launches0, "clocks": clocks}), flush=True)
+
+
 # ----------------------------------------------------------------------------- CUDA arm
 def main():
     args = parse_args()
@@ -342,6 +422,10 @@ def main():
     status = lava.lava_poll_status(plan.workspace)
     if status != 0:
         raise SystemExit("device status word %d after warm-up" % status)
+
+    if args.path != "evict":
+        run_next_path(args, cfg, plan, q, k, v, stream, steps, warmup, local_rank, rank, world)
+        return
 
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
     sampler = ClockSampler(visible_gpu_index(local_rank))

@@ -554,6 +554,10 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     };
 
     // ---- cursors over the CTA's chunks of both passes ---------------------------------------
+    // the order rule compares (pass-1 slot) * S2 with (pass-2 slot + lead) * S1; both sides are
+    // kept as running sums so that a step costs an addition
+    const long long sched1 = m->sched_total1, sched2 = m->sched_total2;
+    long long ord1 = 0, ord2 = (long long)m->lead_tiles * sched1;
     int c1 = blockIdx.x, t1 = 0, last1 = 0;
     long long n1 = 0, j1 = 0;
     bool has1 = c1 < total1;
@@ -590,6 +594,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           z = 0.f;
           ++j1;
           c1 += gridDim.x;
+          ord1 += (long long)(p.chunk_tiles - t1) * sched2;  // the next chunk starts a new run of slots
           t1 = 0;
           has1 = c1 < total1;
           if (has1) open1();
@@ -598,6 +603,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         if ((int)(n1 & 1) == grp) break;
         ++t1;  // the other group's tile
         ++n1;
+        ord1 += sched2;
       }
       // ---- the same for pass 2 ----------------------------------------------------------------
       while (has2 && alive) {
@@ -619,6 +625,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
           prepped = false;
           ++j2;
           c2 += gridDim.x;
+          ord2 += (long long)(p.chunk_tiles - t2) * sched1;
           t2 = 0;
           has2 = c2 < total2;
           if (has2) k2 = decode_chunk(p, m, c2, 2);
@@ -627,13 +634,12 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         if ((int)(n2 & 1) == grp) break;
         ++t2;
         ++n2;
+        ord2 += sched1;
       }
       if (!alive || (!has1 && !has2)) break;
 
       bool take1 = has1;
-      if (has1 && has2)
-        take1 = (j1 * p.chunk_tiles + t1) * (long long)m->sched_total2 <=
-                (j2 * p.chunk_tiles + t2 + m->lead_tiles) * (long long)m->sched_total1;
+      if (has1 && has2) take1 = ord1 <= ord2;
 
       if (take1) {
         // ---- a pass-1 tile: running softmax statistics of 128 keys ------------------------------
@@ -698,6 +704,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         if (lane == 0) mbar_arrive(smem_u32(&m->s1_empty[grp]));
         ++t1;
         ++n1;
+        ord1 += sched2;
       } else {
         // ---- a pass-2 tile: scores of 128 - 2 * pool_radius keys --------------------------------
         if (!prepped) {
@@ -815,6 +822,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         }
         ++t2;
         ++n2;
+        ord2 += sched1;
       }
     }
   } else if (warp >= 12 && warp < 12 + kVWarps) {
