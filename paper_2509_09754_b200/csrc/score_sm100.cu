@@ -558,8 +558,11 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     // kept as running sums so that a step costs an addition
     const long long sched1 = m->sched_total1, sched2 = m->sched_total2;
     long long ord1 = 0, ord2 = (long long)m->lead_tiles * sched1;
-    int c1 = blockIdx.x, t1 = 0, last1 = 0;
-    long long n1 = 0, j1 = 0;
+    // Tile n of a pass (counted over the CTA) belongs to group n & 1, so a group's own tiles are
+    // two apart: t is the index of its next own tile inside the open chunk (it may point past the
+    // chunk's end, into a later chunk), n the tile's number in the CTA.
+    int c1 = blockIdx.x, t1 = grp, n1 = grp, j1 = 0, last1 = 0;
+    ord1 += grp * sched2;
     bool has1 = c1 < total1;
     Chunk k1;
     float mx = -INFINITY, z = 0.f;
@@ -569,72 +572,58 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
       last1 = row < k1.group * W ? min(k1.s.n, k1.s.prefix + t_in_win + 1) : 0;
     };
     if (has1) open1();
-    int c2 = blockIdx.x, t2 = 0;
-    long long n2 = 0, j2 = 0;
+    int c2 = blockIdx.x, t2 = grp, n2 = grp, j2 = 0;
+    ord2 += grp * sched1;
     bool has2 = c2 < total2, prepped = false;
     Chunk k2;
     float es = 0.f, et = 0.f;  // entropy sums of this thread's keys over the chunk
     if (has2) k2 = decode_chunk(p, m, c2, 2);
 
     while (alive) {
-      // ---- move the pass-1 cursor to this group's next tile; close finished chunks ----------
-      while (has1 && alive) {
-        if (t1 == k1.ntiles) {
-          // hand the chunk's statistics (as one log2-sum-exp) to the publisher warp
-          const int slot = (int)(j1 & 1);
-          if (!__all_sync(0xffffffffu, wait_bar(smem_u32(&m->pub_empty[slot]),
-                                                (uint32_t)((j1 >> 1) & 1) ^ 1, m, p.status))) {
-            alive = false;
-            break;
-          }
-          m->pub[slot][grp][row] = z > 0.f ? mx + fast_log2(z) : -INFINITY;
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&m->pub_full[slot]));
-          mx = -INFINITY;
-          z = 0.f;
-          ++j1;
-          c1 += gridDim.x;
-          ord1 += (long long)(p.chunk_tiles - t1) * sched2;  // the next chunk starts a new run of slots
-          t1 = 0;
-          has1 = c1 < total1;
-          if (has1) open1();
-          continue;
+      // ---- close the pass-1 chunks that lie before this group's next tile ---------------------
+      while (has1 && t1 >= k1.ntiles) {
+        // hand the chunk's statistics (as one log2-sum-exp) to the publisher warp
+        const int slot = j1 & 1;
+        if (!__all_sync(0xffffffffu, wait_bar(smem_u32(&m->pub_empty[slot]),
+                                              (uint32_t)((j1 >> 1) & 1) ^ 1, m, p.status))) {
+          alive = false;
+          break;
         }
-        if ((int)(n1 & 1) == grp) break;
-        ++t1;  // the other group's tile
-        ++n1;
-        ord1 += sched2;
+        m->pub[slot][grp][row] = z > 0.f ? mx + fast_log2(z) : -INFINITY;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&m->pub_full[slot]));
+        mx = -INFINITY;
+        z = 0.f;
+        ++j1;
+        c1 += gridDim.x;
+        ord1 += (long long)(p.chunk_tiles - k1.ntiles) * sched2;  // the next chunk starts a new run of slots
+        t1 -= k1.ntiles;
+        has1 = c1 < total1;
+        if (has1) open1();
       }
       // ---- the same for pass 2 ----------------------------------------------------------------
-      while (has2 && alive) {
-        if (t2 == k2.ntiles) {
-          // entropy sums of the chunk in a fixed order: keys of a thread, lanes of a warp; the
-          // eight warp sums of a chunk are added up, in order, by the finishing kernel
+      while (alive && has2 && t2 >= k2.ntiles) {
+        // entropy sums of the chunk in a fixed order: keys of a thread, lanes of a warp; the
+        // eight warp sums of a chunk are added up, in order, by the finishing kernel
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            es += __shfl_down_sync(0xffffffffu, es, o);
-            et += __shfl_down_sync(0xffffffffu, et, o);
-          }
-          if (lane == 0) {
-            p.ent_part[((size_t)k2.head * p.cph2_max + k2.index) * 8 + grp * 4 + quad] =
-                make_float2(es, et);
-            mbar_arrive(smem_u32(&m->prep_empty[j2 & 1]));
-          }
-          es = 0.f;
-          et = 0.f;
-          prepped = false;
-          ++j2;
-          c2 += gridDim.x;
-          ord2 += (long long)(p.chunk_tiles - t2) * sched1;
-          t2 = 0;
-          has2 = c2 < total2;
-          if (has2) k2 = decode_chunk(p, m, c2, 2);
-          continue;
+        for (int o = 16; o > 0; o >>= 1) {
+          es += __shfl_down_sync(0xffffffffu, es, o);
+          et += __shfl_down_sync(0xffffffffu, et, o);
         }
-        if ((int)(n2 & 1) == grp) break;
-        ++t2;
-        ++n2;
-        ord2 += sched1;
+        if (lane == 0) {
+          p.ent_part[((size_t)k2.head * p.cph2_max + k2.index) * 8 + grp * 4 + quad] =
+              make_float2(es, et);
+          mbar_arrive(smem_u32(&m->prep_empty[j2 & 1]));
+        }
+        es = 0.f;
+        et = 0.f;
+        prepped = false;
+        ++j2;
+        c2 += gridDim.x;
+        ord2 += (long long)(p.chunk_tiles - k2.ntiles) * sched1;
+        t2 -= k2.ntiles;
+        has2 = c2 < total2;
+        if (has2) k2 = decode_chunk(p, m, c2, 2);
       }
       if (!alive || (!has1 && !has2)) break;
 
@@ -702,9 +691,9 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         tc_fence_before();
         __syncwarp();  // every lane has finished reading the accumulator
         if (lane == 0) mbar_arrive(smem_u32(&m->s1_empty[grp]));
-        ++t1;
-        ++n1;
-        ord1 += sched2;
+        t1 += 2;
+        n1 += 2;
+        ord1 += 2 * sched2;
       } else {
         // ---- a pass-2 tile: scores of 128 - 2 * pool_radius keys --------------------------------
         if (!prepped) {
@@ -820,9 +809,9 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
             et += sc * __logf(sc);
           }
         }
-        ++t2;
-        ++n2;
-        ord2 += sched1;
+        t2 += 2;
+        n2 += 2;
+        ord2 += 2 * sched1;
       }
     }
   } else if (warp >= 12 && warp < 12 + kVWarps) {
