@@ -153,8 +153,11 @@ __device__ inline Chunk decode_chunk(const Sm100Params& p, const Misc* m, int c,
   ck.group = p.split ? (ck.half ? p.g.group - p.g0 : p.g0) : p.g.group;
   ck.q0 = ck.kvh * p.g.group + ck.half * p.g0;
   ck.s = seq_info(p.g, ck.b);
-  ck.tile0 = ck.index * p.chunk_tiles;
-  ck.ntiles = min(p.chunk_tiles, tiles_of(p, ck.s, pass) - ck.tile0);
+  // the head's tiles are spread evenly over its chunks (none longer than chunk_tiles): a short
+  // last chunk would leave the CTAs with unequal loads
+  const long long tiles = tiles_of(p, ck.s, pass);
+  ck.tile0 = (int)(ck.index * tiles / ck.cph);
+  ck.ntiles = (int)((ck.index + 1) * tiles / ck.cph) - ck.tile0;
   return ck;
 }
 
@@ -1040,7 +1043,7 @@ size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 // balance (chunks are dealt round-robin), and a head finishes pass 1 sooner when more CTAs
 // share it.  Default: about twelve chunks per CTA, between 4 and 32 tiles.  LAVA_SM100_CHUNK_TILES
 // overrides it (option "score_chunk_tiles").
-constexpr int kMinChunkTiles = 4, kMaxChunkTiles = 32;
+constexpr int kMinChunkTiles = 4, kMaxChunkTiles = 64;
 
 // Query groups of more than 128 window-query rows are scored as two halves (each a unit of its
 // own with at most 128 rows); returns the number of query heads in the first half, 0 if the
@@ -1053,7 +1056,11 @@ int chunk_tiles_for(const Geom& g, int n_layers) {
   const long long tiles = (long long)n_layers * (g.n_kv_heads << (sm100_first_half(g) ? 1 : 0)) *
                           ceil_div((int)g.total_tokens, kTile);
   const int sms = sm_count() > 0 ? sm_count() : 148;  // without a device: the part this is tuned for
-  const long long r = tiles / ((long long)sms * 12);
+  // at least four chunks per CTA, and at least three chunks in a sequence of average length (a
+  // batch of short sequences would otherwise be dealt in a few unequal pieces)
+  long long r = tiles / ((long long)sms * 4);
+  const long long mean_tiles = ceil_div((int)(g.total_tokens / g.batch), kTile);
+  if (r > mean_tiles / 3) r = mean_tiles / 3;
   return (int)(r < kMinChunkTiles ? kMinChunkTiles : r > kMaxChunkTiles ? kMaxChunkTiles : r);
 }
 
