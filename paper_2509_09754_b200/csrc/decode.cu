@@ -8,12 +8,11 @@
 //
 // bf16, d = 128: one warp takes up to 512 rows of one (layer, sequence, KV head) for all the
 // head's queries at once and keeps a running (max, sum, output) in the base-2 domain; the
-// partial results of a head's warps are folded by a second small kernel.  K rows go straight
-// from global memory into the B fragments of mma.sync m16n8k16 (S = Q K^T with the queries
-// padded to 16 rows; the order of a dot product's terms is free, so every thread loads whole
-// 16-byte pieces and the query fragments are laid out to match), V rows are staged in shared
-// memory with cp.async (three stages, XOR-swizzled 16-byte pieces) and read with
-// ldmatrix.trans for O += P V.  Other geometries take a plain CUDA-core kernel.
+// partial results of a head's warps are folded by a second small kernel.  K and V rows are
+// staged per warp in shared memory with cp.async (three stages of 16 rows each, XOR-swizzled
+// 16-byte pieces: two tiles are in flight while one is consumed) and read with ldmatrix for
+// mma.sync m16n8k16: S = Q K^T with the queries padded to the 16 rows of the A operand, then
+// O += P V with V read transposed.  Other geometries take a plain CUDA-core kernel.
 #include "sm100_ptx.cuh"
 
 namespace lava {
@@ -55,12 +54,26 @@ __device__ inline uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// Four 8 x 8 matrices of 16-bit elements from shared memory, as stored: thread (g = lane / 4,
+// t = lane % 4) receives elements 2t, 2t+1 of row g of each matrix.
+__device__ inline void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
+                                   uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(saddr)
+               : "memory");
+}
+
+constexpr int kTileBytes = kBlk * 256;              // 16 rows of K or of V
+constexpr int kStageBytes = 2 * kTileBytes;         // K tile, then V tile
+constexpr int kSmemBytes = kWarps * kStages * kStageBytes;
+
 __global__ void __launch_bounds__(kWarps * 32)
 decode_partial_kernel(const DecodeParams p) {
-  __shared__ __align__(128) unsigned char vbuf[kWarps][kStages][kBlk * 256];
+  extern __shared__ __align__(128) unsigned char stage_mem[];
   const Geom& g = p.g;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qrow = lane >> 2, t = lane & 3;  // query row / key row of the fragments, and column pair
+  const int qrow = lane >> 2, t = lane & 3;  // row and column pair of the MMA fragments
   const int prob = blockIdx.z, kvh = blockIdx.y;
   const int chunk = blockIdx.x * kWarps + warp;
   const int* hoff = p.head_offsets + (size_t)prob * (g.n_kv_heads + 1);
@@ -71,67 +84,69 @@ decode_partial_kernel(const DecodeParams p) {
   const long long row0 = p.row_off[prob] + h0 + c0;
   const char* krow = p.k_rows + row0 * 256;
   const char* vrow = p.v_rows + row0 * 256;
+  const uint32_t sbase = smem_u32(stage_mem) + warp * (kStages * kStageBytes);
 
-  // query fragments: rows 0..G-1 of the 16-row A operand hold the head's queries, the rest zeros
-  uint4 qf[4];
+  // query fragments (A operand, 16 x 16 per k-step): rows 0..G-1 hold the head's queries
+  uint32_t qa[8][2];
 #pragma unroll
-  for (int j = 0; j < 4; ++j) qf[j] = make_uint4(0, 0, 0, 0);
+  for (int s = 0; s < 8; ++s) qa[s][0] = qa[s][1] = 0u;
   if (qrow < g.group) {
     const char* qh = (const char*)p.q + ((size_t)prob * g.n_q_heads + kvh * g.group + qrow) * 256;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) qf[j] = *reinterpret_cast<const uint4*>(qh + (t + 4 * j) * 16);
+    for (int s = 0; s < 8; ++s) {
+      qa[s][0] = *reinterpret_cast<const uint32_t*>(qh + (16 * s + 2 * t) * 2);
+      qa[s][1] = *reinterpret_cast<const uint32_t*>(qh + (16 * s + 8 + 2 * t) * 2);
+    }
   }
   const int nblk = (nkeys + kBlk - 1) / kBlk;
-  // V stage fill: 16 rows x 16 pieces, lane l takes pieces l, l+32, ... (row = i / 16)
-  auto fill_v = [&](int blk, int stage) {
-    const uint32_t sbase = smem_u32(&vbuf[warp][stage][0]);
+  // one stage = 16 K rows and 16 V rows, 16-byte pieces XOR-swizzled by the row; rows past the
+  // end are filled with zeros
+  auto fill = [&](int blk, int stage) {
+    const uint32_t st = sbase + stage * kStageBytes;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int idx = lane + 32 * i, r = idx >> 4, pc = idx & 15;
       const int key = blk * kBlk + r;
       const bool ok = key < nkeys;
-      cp_async16(sbase + r * 256 + ((pc ^ (r & 7)) << 4), vrow + (long long)(ok ? key : 0) * 256 + pc * 16, ok);
-    }
-  };
-  // K fragments of a block: pieces t, t+4, t+8, t+12 of rows qrow and qrow + 8 (zeros past the end)
-  auto load_k = [&](uint4 (&kf)[2][4], int blk) {
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-      const int key = blk * kBlk + nt * 8 + qrow;
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        kf[nt][j] = key < nkeys ? ld_stream16(krow + (long long)key * 256 + (t + 4 * j) * 16)
-                                : make_uint4(0, 0, 0, 0);
+      const long long off = (long long)(ok ? key : 0) * 256 + pc * 16;
+      const uint32_t dst = st + r * 256 + ((pc ^ (r & 7)) << 4);
+      cp_async16(dst, krow + off, ok);
+      cp_async16(dst + kTileBytes, vrow + off, ok);
     }
   };
 #pragma unroll
   for (int s = 0; s < kStages - 1; ++s) {
-    if (s < nblk) fill_v(s, s);
+    if (s < nblk) fill(s, s);
     cp_async_commit();
   }
-  uint4 kcur[2][4], knext[2][4];
-  load_k(kcur, 0);
 
   float o[16][4];
 #pragma unroll
   for (int nd = 0; nd < 16; ++nd) o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f;
   float m_run = -INFINITY, l_run = 0.f;
   const float sc2 = g.scale_log2;
+  const int mi = lane >> 3, r8 = lane & 7;
 
   for (int blk = 0; blk < nblk; ++blk) {
-    if (blk + kStages - 1 < nblk) fill_v(blk + kStages - 1, (blk + kStages - 1) % kStages);
+    if (blk + kStages - 1 < nblk) fill(blk + kStages - 1, (blk + kStages - 1) % kStages);
     cp_async_commit();
-    if (blk + 1 < nblk) load_k(knext, blk + 1);
-    // ---- S = Q K^T for 16 rows: two 8-key tiles, eight k-steps each ---------------------------
+    cp_async_wait<kStages - 1>();
+    __syncwarp();
+    const uint32_t st = sbase + (blk % kStages) * kStageBytes;
+    // ---- S = Q K^T for 16 rows: two 8-key tiles, eight k-steps --------------------------------
     float s[2][4];
+    s[0][0] = s[0][1] = s[0][2] = s[0][3] = 0.f;
+    s[1][0] = s[1][1] = s[1][2] = s[1][3] = 0.f;
+    {
+      // matrices of one k-step: (keys 0-7, piece 2s), (keys 0-7, piece 2s+1), (keys 8-15, ...)
+      const int key_l = (mi >> 1) * 8 + r8;
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint4 a = qf[j], b = kcur[nt][j];
-        mma_bf16_16816(s[nt][0], s[nt][1], s[nt][2], s[nt][3], a.x, 0u, a.y, 0u, b.x, b.y);
-        mma_bf16_16816(s[nt][0], s[nt][1], s[nt][2], s[nt][3], a.z, 0u, a.w, 0u, b.z, b.w);
+      for (int ks = 0; ks < 8; ++ks) {
+        uint32_t b0, b1, b2, b3;
+        const int pc = 2 * ks + (mi & 1);
+        ldmatrix_x4(b0, b1, b2, b3, st + key_l * 256 + ((pc ^ (key_l & 7)) << 4));
+        mma_bf16_16816(s[0][0], s[0][1], s[0][2], s[0][3], qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+        mma_bf16_16816(s[1][0], s[1][1], s[1][2], s[1][3], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
       }
     }
     // ---- running softmax of query row qrow over its keys 2t, 2t+1 (+8) --------------------------
@@ -160,23 +175,18 @@ decode_partial_kernel(const DecodeParams p) {
     }
     const uint32_t pa0 = pack_bf16(pr[0], pr[1]), pa2 = pack_bf16(pr[2], pr[3]);
     // ---- O += P V ----------------------------------------------------------------------------
-    cp_async_wait<kStages - 1>();
-    __syncwarp();
-    const uint32_t sbase = smem_u32(&vbuf[warp][blk % kStages][0]);
-    const int mi = lane >> 3, key_l = (mi & 1) * 8 + (lane & 7);
+    {
+      const int key_l = (mi & 1) * 8 + r8;
 #pragma unroll
-    for (int nd = 0; nd < 16; nd += 2) {
-      uint32_t b0, b1, b2, b3;
-      const int pc = nd + (mi >> 1);
-      ldmatrix_x4_trans(b0, b1, b2, b3, sbase + key_l * 256 + ((pc ^ (key_l & 7)) << 4));
-      mma_bf16_16816(o[nd][0], o[nd][1], o[nd][2], o[nd][3], pa0, 0u, pa2, 0u, b0, b1);
-      mma_bf16_16816(o[nd + 1][0], o[nd + 1][1], o[nd + 1][2], o[nd + 1][3], pa0, 0u, pa2, 0u, b2, b3);
+      for (int nd = 0; nd < 16; nd += 2) {
+        uint32_t b0, b1, b2, b3;
+        const int pc = nd + (mi >> 1);
+        ldmatrix_x4_trans(b0, b1, b2, b3, st + kTileBytes + key_l * 256 + ((pc ^ (key_l & 7)) << 4));
+        mma_bf16_16816(o[nd][0], o[nd][1], o[nd][2], o[nd][3], pa0, 0u, pa2, 0u, b0, b1);
+        mma_bf16_16816(o[nd + 1][0], o[nd + 1][1], o[nd + 1][2], o[nd + 1][3], pa0, 0u, pa2, 0u, b2, b3);
+      }
     }
     __syncwarp();  // the stage may be refilled by the next iteration
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) kcur[nt][j] = knext[nt][j];
   }
   cp_async_wait<0>();
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
@@ -322,7 +332,19 @@ lava_status lava_decode_attention_layers(const lava_layer_desc* desc, int32_t n_
   if (!aligned16(workspace)) return fail(LAVA_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
   p.part = (float*)workspace;
   dim3 grid((p.chunks_max + kWarps - 1) / kWarps, g.n_kv_heads, n_layers * g.batch);
-  decode_partial_kernel<<<grid, kWarps * 32, 0, st>>>(p);
+  {
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+      rc = check_cuda(cudaFuncSetAttribute(decode_partial_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
+                      "decode attention attribute");
+      if (rc != LAVA_OK) return rc;
+      configured[dev] = true;
+    }
+  }
+  decode_partial_kernel<<<grid, kWarps * 32, kSmemBytes, st>>>(p);
   decode_combine_kernel<<<dim3(g.n_q_heads, n_layers * g.batch), 128, 0, st>>>(p);
   count_launches(2);
   return check_cuda(cudaGetLastError(), "decode attention launch");
