@@ -580,7 +580,14 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
     bool has2 = c2 < total2, prepped = false;
     Chunk k2;
     float es = 0.f, et = 0.f;  // entropy sums of this thread's keys over the chunk
-    if (has2) k2 = decode_chunk(p, m, c2, 2);
+    float* dst_head = nullptr;   // score row of the open chunk's KV head
+    float chunk_scale = 0.f;     // Vbar * c_hat of that head
+    auto open2 = [&]() {
+      k2 = decode_chunk(p, m, c2, 2);
+      dst_head = p.scores + (size_t)k2.layer * g.total_scores + k2.s.score_off +
+                 (long long)k2.kvh * k2.s.prefix;
+    };
+    if (has2) open2();
 
     while (alive) {
       // ---- close the pass-1 chunks that lie before this group's next tile ---------------------
@@ -626,7 +633,7 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
         ord2 += (long long)(p.chunk_tiles - k2.ntiles) * sched1;
         t2 -= k2.ntiles;
         has2 = c2 < total2;
-        if (has2) k2 = decode_chunk(p, m, c2, 2);
+        if (has2) open2();
       }
       if (!alive || (!has1 && !has2)) break;
 
@@ -704,11 +711,11 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
                                                 (uint32_t)((j2 >> 1) & 1), m, p.status)))
             break;
           prepped = true;
+          chunk_scale = m->prep[j2 & 1].scale;
         }
         if (!__all_sync(0xffffffffu, wait_bar(smem_u32(&m->s2_full[grp]),
                                               (uint32_t)((n2 >> 1) & 1), m, p.status)))
           break;
-        const Prep* prep = &m->prep[j2 & 1];
         const int tile = k2.tile0 + t2;
         tc_fence_after();
         float acc[NH];
@@ -800,9 +807,8 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
               for (int q = 1; q <= rad; ++q) best = fmaxf(best, fmaxf(a[-q], a[q]));
             }
           }
-          const float sc = best * prep->scale;
-          float* dst = p.scores + (size_t)k2.layer * g.total_scores + k2.s.score_off +
-                       (long long)k2.kvh * k2.s.prefix + i;
+          const float sc = best * chunk_scale;
+          float* dst = dst_head + i;
           // split mode: the group maximum over the two halves is taken in memory (scores are
           // >= 0, so their bit patterns order like the values; the array starts as zeros)
           if (p.split) atomicMax(reinterpret_cast<unsigned*>(dst), __float_as_uint(sc));
