@@ -12,7 +12,9 @@
 // staged per warp in shared memory with cp.async (three stages of 16 rows each, XOR-swizzled
 // 16-byte pieces: two tiles are in flight while one is consumed) and read with ldmatrix for
 // mma.sync m16n8k16: S = Q K^T with the queries padded to the 16 rows of the A operand, then
-// O += P V with V read transposed.  Other geometries take a plain CUDA-core kernel.
+// O += P V with V read transposed.  The (head, chunk) pairs that have rows are listed by a small
+// kernel first, and a fixed grid of warps walks that list.  Other geometries take a plain
+// CUDA-core kernel.
 #include "sm100_ptx.cuh"
 
 namespace lava {
@@ -35,7 +37,9 @@ struct DecodeParams {
   const long long* row_off; // [layers * batch (+1)]
   float* part;              // [layers*batch*H_kv][chunks_max][group][kPartStride]
   float* out;               // [layers, batch, H_q, d]
-  int chunks_max;
+  int2* items;              // work list: (head = prob * H_kv + kvh, chunk) of every non-empty chunk
+  int* n_items;
+  int chunks_max, heads;
 };
 
 __device__ inline void cp_async16(uint32_t saddr, const void* src, bool valid) {
@@ -68,18 +72,60 @@ constexpr int kTileBytes = kBlk * 256;              // 16 rows of K or of V
 constexpr int kStageBytes = 2 * kTileBytes;         // K tile, then V tile
 constexpr int kSmemBytes = kWarps * kStages * kStageBytes;
 
+// Row counts live on the device, so the list of (head, chunk) pairs that have rows is built
+// there: one block walks the heads in order (exclusive scan of their chunk counts) and writes
+// the pairs; the attention kernel then runs a fixed grid over that list and no CTA is launched
+// for nothing.
+__global__ void __launch_bounds__(1024)
+decode_plan_kernel(const DecodeParams p) {
+  __shared__ int wsum[32];
+  __shared__ int base;
+  const Geom& g = p.g;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int h0 = 0; h0 < p.heads; h0 += 1024) {
+    const int h = h0 + threadIdx.x;
+    int cnt = 0;
+    if (h < p.heads) {
+      const int prob = h / g.n_kv_heads, kvh = h - prob * g.n_kv_heads;
+      const int* hoff = p.head_offsets + (size_t)prob * (g.n_kv_heads + 1);
+      const int len = hoff[kvh + 1] - hoff[kvh];
+      cnt = len > 0 ? min((len + kChunk - 1) / kChunk, p.chunks_max) : 0;
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    int before = base;
+    for (int wdx = 0; wdx < warp; ++wdx) before += wsum[wdx];
+    const int start = before + incl - cnt;
+    for (int c = 0; c < cnt; ++c) p.items[start + c] = make_int2(h, c);
+    __syncthreads();
+    if (threadIdx.x == 1023) base = start + cnt;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *p.n_items = base;
+}
+
 __global__ void __launch_bounds__(kWarps * 32)
 decode_partial_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) unsigned char stage_mem[];
   const Geom& g = p.g;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qrow = lane >> 2, t = lane & 3;  // row and column pair of the MMA fragments
-  const int prob = blockIdx.z, kvh = blockIdx.y;
-  const int chunk = blockIdx.x * kWarps + warp;
+  const int n_items = *p.n_items;
+  for (int item = blockIdx.x * kWarps + warp; item < n_items; item += gridDim.x * kWarps) {
+  const int2 it = p.items[item];
+  const int prob = it.x / g.n_kv_heads, kvh = it.x - prob * g.n_kv_heads;
+  const int chunk = it.y;
   const int* hoff = p.head_offsets + (size_t)prob * (g.n_kv_heads + 1);
   const int h0 = hoff[kvh], len = hoff[kvh + 1] - h0;
   const int c0 = chunk * kChunk;
-  if (c0 >= len) return;  // whole warp
   const int nkeys = min(kChunk, len - c0);
   const long long row0 = p.row_off[prob] + h0 + c0;
   const char* krow = p.k_rows + row0 * 256;
@@ -202,6 +248,8 @@ decode_partial_kernel(const DecodeParams p) {
       dst[129] = l_run;
     }
   }
+  __syncwarp();  // the stages are refilled by the warp's next item
+  }
 }
 
 // Fold of a head's partial results, in chunk order.
@@ -276,9 +324,14 @@ decode_generic_kernel(const DecodeParams p) {
   if (tid < d) p.out[((size_t)prob * g.n_q_heads + h) * d + tid] = len > 0 ? acc / l : 0.f;
 }
 
+inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 inline size_t part_bytes(const Geom& g, int n_layers) {
   const size_t chunks_max = (size_t)(g.max_seqlen + kChunk - 1) / kChunk;
-  return (size_t)n_layers * g.batch * g.n_kv_heads * chunks_max * g.group * kPartStride * sizeof(float);
+  return up256((size_t)n_layers * g.batch * g.n_kv_heads * chunks_max * g.group * kPartStride * sizeof(float));
+}
+inline size_t item_bytes(const Geom& g, int n_layers) {
+  const size_t chunks_max = (size_t)(g.max_seqlen + kChunk - 1) / kChunk;
+  return up256((size_t)n_layers * g.batch * g.n_kv_heads * chunks_max * sizeof(int2));
 }
 
 }  // namespace
@@ -291,7 +344,7 @@ extern "C" {
 size_t lava_decode_workspace_bytes(const lava_layer_desc* desc, int32_t n_layers) {
   Geom g;
   if (n_layers < 1 || make_geom(desc, &g) != LAVA_OK) return 0;
-  return part_bytes(g, n_layers) + 256;
+  return part_bytes(g, n_layers) + item_bytes(g, n_layers) + 256;
 }
 
 lava_status lava_decode_attention_layers(const lava_layer_desc* desc, int32_t n_layers, const void* q,
@@ -318,7 +371,10 @@ lava_status lava_decode_attention_layers(const lava_layer_desc* desc, int32_t n_
   p.row_off = (const long long*)layer_row_offset;
   p.out = out;
   p.part = nullptr;
+  p.items = nullptr;
+  p.n_items = nullptr;
   p.chunks_max = (g.max_seqlen + kChunk - 1) / kChunk;
+  p.heads = n_layers * g.batch * g.n_kv_heads;
   cudaStream_t st = (cudaStream_t)stream;
   const bool tensor_path = g.dtype == LAVA_BF16 && g.head_dim == 128 && g.group <= 8;
   if (!tensor_path) {
@@ -326,12 +382,18 @@ lava_status lava_decode_attention_layers(const lava_layer_desc* desc, int32_t n_
     count_launches(1);
     return check_cuda(cudaGetLastError(), "decode attention launch");
   }
-  const size_t need = part_bytes(g, n_layers);
+  const size_t need = part_bytes(g, n_layers) + item_bytes(g, n_layers) + 256;
   if (!workspace || workspace_bytes < need)
     return fail(LAVA_ERR_WORKSPACE, "workspace too small: %zu < %zu bytes", workspace_bytes, need);
   if (!aligned16(workspace)) return fail(LAVA_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
   p.part = (float*)workspace;
-  dim3 grid((p.chunks_max + kWarps - 1) / kWarps, g.n_kv_heads, n_layers * g.batch);
+  p.items = (int2*)((char*)workspace + part_bytes(g, n_layers));
+  p.n_items = (int*)((char*)workspace + part_bytes(g, n_layers) + item_bytes(g, n_layers));
+  decode_plan_kernel<<<1, 1024, 0, st>>>(p);
+  // two CTAs fit an SM (shared memory); a few CTAs per slot even out items of unequal length
+  const long long slots = (long long)(sm_count() > 0 ? sm_count() : 1) * 2;
+  const long long max_items = (long long)p.heads * p.chunks_max;
+  const int grid = (int)std::max<long long>(1, std::min(slots, (max_items + kWarps - 1) / kWarps));
   {
     static bool configured[64] = {};
     int dev = 0;
@@ -346,7 +408,7 @@ lava_status lava_decode_attention_layers(const lava_layer_desc* desc, int32_t n_
   }
   decode_partial_kernel<<<grid, kWarps * 32, kSmemBytes, st>>>(p);
   decode_combine_kernel<<<dim3(g.n_q_heads, n_layers * g.batch), 128, 0, st>>>(p);
-  count_launches(2);
+  count_launches(3);
   return check_cuda(cudaGetLastError(), "decode attention launch");
 }
 

@@ -1050,6 +1050,7 @@ size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 // share it.  Default: about twelve chunks per CTA, between 4 and 32 tiles.  LAVA_SM100_CHUNK_TILES
 // overrides it (option "score_chunk_tiles").
 constexpr int kMinChunkTiles = 4, kMaxChunkTiles = 64;
+constexpr int kSmallLaunchChunkTiles = 8;  // floor of the chosen length: shorter chunks cost more in boundaries than they balance
 
 // Query groups of more than 128 window-query rows are scored as two halves (each a unit of its
 // own with at most 128 rows); returns the number of query heads in the first half, 0 if the
@@ -1067,6 +1068,7 @@ int chunk_tiles_for(const Geom& g, int n_layers) {
   long long r = tiles / ((long long)sms * 4);
   const long long mean_tiles = ceil_div((int)(g.total_tokens / g.batch), kTile);
   if (r > mean_tiles / 3) r = mean_tiles / 3;
+  if (r < kSmallLaunchChunkTiles) r = mean_tiles < kSmallLaunchChunkTiles ? mean_tiles : kSmallLaunchChunkTiles;
   return (int)(r < kMinChunkTiles ? kMinChunkTiles : r > kMaxChunkTiles ? kMaxChunkTiles : r);
 }
 
