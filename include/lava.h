@@ -354,6 +354,52 @@ LAVA_API lava_status lava_decode_attention(const lava_layer_desc* desc, const vo
                                            const int64_t* layer_row_offset, float* out,
                                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* Layer-wide selection (Algorithm 1, Evict) with the KV heads of a layer split over several GPUs.
+ * Every rank describes its own heads (desc->n_kv_heads = local heads, scores of the local heads in
+ * the usual layout) and the ranks agree on one threshold per (layer, sequence).  The library
+ * provides the local steps; the caller runs the two small collectives between them:
+ *
+ *   lava_select_shard_begin(desc, L, total_kv_heads, layer_budget, state)
+ *   for pass in 0, 1, 2:
+ *       lava_select_shard_hist(desc, L, scores, pass, state)     -- fills the histogram block
+ *       all-reduce (sum, uint32) of the histogram block over the ranks
+ *       lava_select_shard_step(desc, L, pass, state)             -- same result on every rank
+ *   lava_select_shard_count(desc, L, scores, state)              -- fills the tie block
+ *   ties_before_rank[p] = sum of the tie blocks of the lower ranks (all-gather + prefix);
+ *                         a separate DEVICE int64 [L*batch] array, zeros on rank 0
+ *   lava_select_shard_emit(desc, L, scores, ties_before_rank, keep_idx, head_offsets,
+ *                          layer_row_offset, state)
+ *
+ * Heads are ordered by rank, then by local index: equal scores go to the lower rank first, so the
+ * union of the ranks' outputs equals lava_select_topk on the unsplit layer.  keep_idx and
+ * head_offsets are local (same layout as lava_select_topk for the local desc); layer_row_offset
+ * (may be NULL) receives the prefix sums of the LOCAL row counts, ready for lava_compact_kv on the
+ * rank's own K/V.  layer_budget is the budget of the whole layer (all ranks pass the same).
+ * `state` is DEVICE memory of lava_select_shard_bytes(desc, L) bytes; lava_select_shard_layout
+ * gives the byte ranges of the histogram block (uint32 [L*batch][2048]) and of the tie block
+ * (int64 [L*batch]) inside it.  No kernel here reads another GPU's memory. */
+LAVA_API size_t lava_select_shard_bytes(const lava_layer_desc* desc, int32_t n_layers);
+LAVA_API lava_status lava_select_shard_layout(const lava_layer_desc* desc, int32_t n_layers,
+                                              size_t* hist_offset, size_t* hist_bytes,
+                                              size_t* ties_offset, size_t* ties_bytes);
+LAVA_API lava_status lava_select_shard_begin(const lava_layer_desc* desc, int32_t n_layers,
+                                             int32_t total_kv_heads, const int64_t* layer_budget,
+                                             void* state, size_t state_bytes, void* stream);
+LAVA_API lava_status lava_select_shard_hist(const lava_layer_desc* desc, int32_t n_layers,
+                                            const float* scores, int32_t pass, void* state,
+                                            size_t state_bytes, void* stream);
+LAVA_API lava_status lava_select_shard_step(const lava_layer_desc* desc, int32_t n_layers,
+                                            int32_t pass, void* state, size_t state_bytes,
+                                            void* stream);
+LAVA_API lava_status lava_select_shard_count(const lava_layer_desc* desc, int32_t n_layers,
+                                             const float* scores, void* state, size_t state_bytes,
+                                             void* stream);
+LAVA_API lava_status lava_select_shard_emit(const lava_layer_desc* desc, int32_t n_layers,
+                                            const float* scores, const int64_t* ties_before_rank,
+                                            int32_t* keep_idx, int32_t* head_offsets,
+                                            int64_t* layer_row_offset, void* state,
+                                            size_t state_bytes, void* stream);
+
 /* Evaluator (not on the eviction path): layer attention output loss of a selection, Lemma 1 with
  * p = 1 for the last token of every sequence, and the upper bound of Theorem 1:
  *     loss[b]  = || Cat_h[ (A_h - A^_h) V_g(h) ] W_O ||_1 ,  A^_h = (A_h (.) I) / ||A_h (.) I||_1

@@ -13,6 +13,8 @@ from .binding import (  # noqa: F401
     lava_score_layer, lava_score_layer_static, lava_score_layers, lava_layer_budgets,
     lava_select_topk, lava_select_topk_layers, lava_compact_kv, lava_compact_kv_layers,
     EvictionPlan, evict_model, lava_layer_output_loss,
+    lava_select_shard_bytes, lava_select_shard_layout, lava_select_shard_begin, lava_select_shard_hist,
+    lava_select_shard_step, lava_select_shard_count, lava_select_shard_emit,
     lava_decode_workspace_bytes, lava_decode_attention_layers, lava_decode_attention, Cascade, lava_cascade_state_bytes,
     lava_launch_count, lava_score_path, lava_set_option, lava_get_option, lava_host_arena_bytes, lava_evict_model_host,
 )

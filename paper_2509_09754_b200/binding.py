@@ -93,6 +93,18 @@ def load_library():
     lib.lava_set_option.argtypes = [ctypes.c_char_p, i64]
     lib.lava_get_option.restype = i64
     lib.lava_get_option.argtypes = [ctypes.c_char_p]
+    lib.lava_select_shard_bytes.restype = sz
+    lib.lava_select_shard_bytes.argtypes = [dp, i32]
+    szp = ctypes.POINTER(sz)
+    lib.lava_select_shard_layout.argtypes = [dp, i32, szp, szp, szp, szp]
+    lib.lava_select_shard_begin.argtypes = [dp, i32, i32, vp, vp, sz, vp]
+    lib.lava_select_shard_hist.argtypes = [dp, i32, vp, i32, vp, sz, vp]
+    lib.lava_select_shard_step.argtypes = [dp, i32, i32, vp, sz, vp]
+    lib.lava_select_shard_count.argtypes = [dp, i32, vp, vp, sz, vp]
+    lib.lava_select_shard_emit.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+    for name in ("lava_select_shard_layout", "lava_select_shard_begin", "lava_select_shard_hist",
+                 "lava_select_shard_step", "lava_select_shard_count", "lava_select_shard_emit"):
+        getattr(lib, name).restype = i32
     lib.lava_decode_workspace_bytes.restype = sz
     lib.lava_decode_workspace_bytes.argtypes = [dp, i32]
     lib.lava_decode_attention_layers.restype = i32
@@ -367,6 +379,47 @@ def evict_model(plan: EvictionPlan, q_win, k, v, mode: int = LAVA_BUDGET_DYNAMIC
     lava_compact_kv_layers(d, nl, k, v, k.stride(0), v.stride(0), plan.keep_idx,
                            plan.head_offsets, plan.layer_row_offset, plan.k_out, plan.v_out,
                            stream)
+
+
+# ----------------------------------------------------------------------------- sharded selection
+def lava_select_shard_bytes(desc: LayerDesc, n_layers: int) -> int:
+    return load_library().lava_select_shard_bytes(ctypes.byref(desc.to_c()), n_layers)
+
+
+def lava_select_shard_layout(desc: LayerDesc, n_layers: int):
+    """(hist_offset, hist_bytes, ties_offset, ties_bytes) inside the shard state block."""
+    v = [ctypes.c_size_t() for _ in range(4)]
+    _check(load_library().lava_select_shard_layout(ctypes.byref(desc.to_c()), n_layers,
+                                                   *[ctypes.byref(x) for x in v]))
+    return tuple(int(x.value) for x in v)
+
+
+def lava_select_shard_begin(desc, n_layers, total_kv_heads, layer_budget, state, stream=None):
+    _check(load_library().lava_select_shard_begin(ctypes.byref(desc.to_c()), n_layers, total_kv_heads,
+                                                  _ptr(layer_budget), _ptr(state), state.numel(),
+                                                  _stream(stream)))
+
+
+def lava_select_shard_hist(desc, n_layers, scores, pass_, state, stream=None):
+    _check(load_library().lava_select_shard_hist(ctypes.byref(desc.to_c()), n_layers, _ptr(scores),
+                                                 pass_, _ptr(state), state.numel(), _stream(stream)))
+
+
+def lava_select_shard_step(desc, n_layers, pass_, state, stream=None):
+    _check(load_library().lava_select_shard_step(ctypes.byref(desc.to_c()), n_layers, pass_,
+                                                 _ptr(state), state.numel(), _stream(stream)))
+
+
+def lava_select_shard_count(desc, n_layers, scores, state, stream=None):
+    _check(load_library().lava_select_shard_count(ctypes.byref(desc.to_c()), n_layers, _ptr(scores),
+                                                  _ptr(state), state.numel(), _stream(stream)))
+
+
+def lava_select_shard_emit(desc, n_layers, scores, ties_before_rank, keep_idx, head_offsets,
+                           layer_row_offset, state, stream=None):
+    _check(load_library().lava_select_shard_emit(
+        ctypes.byref(desc.to_c()), n_layers, _ptr(scores), _ptr(ties_before_rank), _ptr(keep_idx),
+        _ptr(head_offsets), _ptr(layer_row_offset), _ptr(state), state.numel(), _stream(stream)))
 
 
 def lava_decode_workspace_bytes(desc: LayerDesc, n_layers: int = 1) -> int:

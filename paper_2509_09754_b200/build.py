@@ -12,7 +12,7 @@ LIB_DIR = os.path.join(PKG, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "liblava.so")
 
 SOURCES = ["lava_api.cu", "score_generic.cu", "budgets.cu", "select.cu", "compact.cu",
-           "host_path.cu", "score_sm100.cu", "score_tmem.cu", "score_variants.cu", "cascade.cu", "loss_eval.cu", "decode.cu", "score_static.cu"]
+           "host_path.cu", "score_sm100.cu", "score_tmem.cu", "score_variants.cu", "cascade.cu", "loss_eval.cu", "decode.cu", "select_shard.cu", "score_static.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
