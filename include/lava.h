@@ -63,7 +63,10 @@ typedef enum lava_budget_mode {
 } lava_budget_mode;
 
 /* Bits of the device status word. */
-#define LAVA_DEV_SHORT_SEQUENCE 1u    /* some sequence has fewer than `window` tokens        */
+#define LAVA_DEV_SHORT_SEQUENCE 1u    /* some sequence has fewer than `window` tokens: the score
+                                         layout has no room for it, so the score, select and
+                                         compact kernels of such a batch do nothing at all (the
+                                         host can only check total_tokens >= batch*window)      */
 #define LAVA_DEV_BUDGET_INFEASIBLE 2u /* total budget outside [L*floor, L*cap]; was clamped  */
 #define LAVA_DEV_WAIT_EXPIRED 4u      /* a bounded wait inside a kernel gave up              */
 #define LAVA_DEV_BAD_SEQLEN 8u        /* some sequence is longer than desc->max_seqlen       */

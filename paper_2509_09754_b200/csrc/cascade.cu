@@ -92,6 +92,7 @@ __global__ void cascade_init_kernel(Geom g, int n_layers, long long rows, const 
 __global__ void __launch_bounds__(256)
 cascade_adopt_kernel(Geom g, const float* scores_full, const int* keep_full, const int* head_offsets,
                      const long long* row_off, float* score_list, int* pos_list) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   const int b = blockIdx.y;
   const SeqInfo s = seq_info(g, b);
   const int win = min(g.window, s.n);
@@ -113,6 +114,7 @@ __global__ void __launch_bounds__(256)
 cascade_move_kernel(Geom g, const int* src_pos, const int* hoff_old_all, const int* hoff_new_all,
                     const long long* roff_old, const long long* roff_new, const char* k_old,
                     const char* v_old, char* k_new, char* v_new, int blocks_per_head) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   const int prob = blockIdx.z, b = prob % g.batch, kvh = blockIdx.y;
   const SeqInfo s = seq_info(g, b);
   const int win = min(g.window, s.n);

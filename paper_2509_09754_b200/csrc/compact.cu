@@ -13,6 +13,7 @@ __global__ void __launch_bounds__(256)
 compact_kernel(Geom g, const char* k, const char* v, long long k_ls, long long v_ls,
                const int* keep_idx, const int* head_offsets, const long long* row_off,
                char* k_out, char* v_out, int blocks_per_head) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   const int prob = blockIdx.z, layer = prob / g.batch, b = prob - layer * g.batch;
   const int kvh = blockIdx.y;
   const SeqInfo s = seq_info(g, b);

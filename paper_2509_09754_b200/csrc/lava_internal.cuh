@@ -44,6 +44,23 @@ __device__ inline SeqInfo seq_info(const Geom& g, int b) {
   return s;
 }
 
+// The score layout gives sequence b the offset H_kv * (tok0 - b*w): it has no room for a sequence
+// shorter than the window (the host can only check the total, the lengths live on the device).
+// Every kernel that addresses scores or kept positions through that layout asks this first and
+// does nothing if it holds, so that such a batch cannot write outside its arrays; the score
+// kernels also report LAVA_DEV_SHORT_SEQUENCE.  Block-wide: every thread of a one-dimensional
+// block must call it.
+__device__ inline bool batch_has_short_sequence(const Geom& g) {
+  int bad = 0;
+  if (g.cu_seqlens) {
+    for (int b = threadIdx.x; b < g.batch; b += blockDim.x)
+      bad |= (g.cu_seqlens[b + 1] - g.cu_seqlens[b]) < g.window;
+  } else {
+    bad = g.total_tokens < g.window;
+  }
+  return __syncthreads_or(bad) != 0;
+}
+
 // Workspace layout (byte offsets from the workspace base), identical for every caller.
 struct Workspace {
   static constexpr size_t kStatusBytes = 256;

@@ -98,6 +98,7 @@ loss_attention_kernel(Geom g, const void* q_win, const void* k, double* att) {
 // I_g: kept prefix positions and the window.  One block per (KV head, sequence).
 __global__ void __launch_bounds__(256)
 loss_mask_kernel(Geom g, const int* keep_idx, const int* head_offsets, unsigned char* mask) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   const int kvh = blockIdx.x, b = blockIdx.y;
   const SeqInfo s = seq_info(g, b);
   const int win = min(g.window, s.n);

@@ -273,6 +273,7 @@ score_kernel(Geom g, const char* q, const char* k, long long q_ls, long long k_l
   __shared__ float nl[128];
   __shared__ double red_s[kThreads / 32], red_t[kThreads / 32];
 
+  if (batch_has_short_sequence(g)) return;  // reported by the combine kernel
   const int prob = blockIdx.z, layer = prob / g.batch, b = prob - layer * g.batch;
   const int kvh = blockIdx.y, slice = blockIdx.x;
   const SeqInfo s = seq_info(g, b);

@@ -175,6 +175,10 @@ lava_score_sm100_kernel(const __grid_constant__ CUtensorMap map_q,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Geom& g = p.g;
   const int units = g.n_kv_heads << p.split;  // scored units per sequence
+  if (batch_has_short_sequence(g)) {  // every CTA sees the same lengths: all of them leave
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(p.status, LAVA_DEV_SHORT_SEQUENCE);
+    return;
+  }
 
   // ---- chunk schedule: exclusive scans of chunks per sequence, both passes -------------------
   {
@@ -979,6 +983,7 @@ entropy_from_scores_kernel(Geom g, const float* scores, double* entropy, const f
                            const unsigned* vbar_bits, float* vbar_out) {
   __shared__ double rs[32], rt[32];
   const int prob = blockIdx.x, layer = prob / g.batch, b = prob - layer * g.batch;
+  if (batch_has_short_sequence(g)) return;
   const SeqInfo s = seq_info(g, b);
   if (vbar_out && (int)threadIdx.x < g.n_kv_heads) {
     const size_t head = (size_t)prob * g.n_kv_heads + threadIdx.x;

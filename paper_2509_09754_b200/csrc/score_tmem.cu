@@ -238,6 +238,10 @@ lava_score_tmem_kernel(const __grid_constant__ CUtensorMap map_q,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Geom& g = p.g;
   const int rad = g.pool_radius, nunit = p.nunit;
+  if (batch_has_short_sequence(g)) {  // every CTA sees the same lengths: all of them leave
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(p.status, LAVA_DEV_SHORT_SEQUENCE);
+    return;
+  }
 
   // ---- tiles per sequence (exclusive scan), barriers, tensor memory ---------------------------
   __shared__ int bad_len;

@@ -21,6 +21,7 @@ __global__ void fill_ones_kernel(float* dst, long long count) {
 // One warp per prefix position of one KV head: the row's L1 norm times the position's score.
 __global__ void __launch_bounds__(256)
 token_norm_scale_kernel(Geom g, const char* v, long long v_ls, float* scores) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   const int prob = blockIdx.z, layer = prob / g.batch, b = prob - layer * g.batch;
   const int kvh = blockIdx.y;
   const SeqInfo s = seq_info(g, b);

@@ -58,6 +58,7 @@ __device__ inline unsigned block_exclusive_scan(unsigned x, unsigned* warp_sum, 
 __global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads)
 select_topk_kernel(Geom g, const float* scores, const long long* layer_budget, int* keep_idx,
                    int* head_offsets) {
+  if (batch_has_short_sequence(g)) return;  // every CTA of the cluster sees the same lengths
   __shared__ SelectShared sh;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -237,6 +238,7 @@ __global__ void __launch_bounds__(kThreads, RegCfg<E>::kMinCtas)
 select_topk_reg_kernel(Geom g, const float* scores, const long long* layer_budget, int* keep_idx,
                        int* head_offsets, HeldLists io) {
   using Cfg = RegCfg<E>;
+  if (batch_has_short_sequence(g)) return;  // every CTA of the cluster sees the same lengths
   extern __shared__ __align__(16) unsigned big[];  // staging / histogram copies / packed output
   __shared__ RegShared sh;
   cg::cluster_group cluster = cg::this_cluster();

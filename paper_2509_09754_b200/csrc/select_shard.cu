@@ -42,6 +42,7 @@ __global__ void shard_begin_kernel(Geom g, int n_layers, int total_kv_heads,
 
 __global__ void __launch_bounds__(512)
 shard_hist_kernel(Geom g, const float* scores, const ShardState* state, int pass, unsigned* hist) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   __shared__ unsigned sh[kBins];
   const int prob = blockIdx.y, layer = prob / g.batch;
   const SeqInfo s = seq_info(g, prob - layer * g.batch);
@@ -117,6 +118,7 @@ shard_step_kernel(int pass, const unsigned* hist, ShardState* state) {
 // counts[prob][head] = (entries above tau, entries equal to tau) of every local head.
 __global__ void __launch_bounds__(512)
 shard_count_kernel(Geom g, const float* scores, const ShardState* state, uint2* counts) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   __shared__ unsigned wg[16], we[16];
   const int prob = blockIdx.y, layer = prob / g.batch, head = blockIdx.x;
   const SeqInfo s = seq_info(g, prob - layer * g.batch);
@@ -165,6 +167,7 @@ __global__ void __launch_bounds__(1024)
 shard_emit_kernel(Geom g, const float* scores, const ShardState* state, const uint2* counts,
                   const long long* ties_before_rank, int* keep_idx, int* head_offsets,
                   long long* rows_out) {
+  if (batch_has_short_sequence(g)) return;  // the score layout has no room for such a batch
   __shared__ unsigned wsum[32];
   __shared__ unsigned run_keep, run_eq;
   const int prob = blockIdx.y, layer = prob / g.batch, head = blockIdx.x;

@@ -155,3 +155,35 @@ def test_cascade_rejects_what_it_does_not_cover_and_steps_out_of_order():
         cas.step(q[1], k[1], v[1])                                       # all layers taken
     torch.cuda.synchronize()
     cas.close()
+
+
+def test_a_sequence_shorter_than_the_window_stops_the_batch():
+    """The score layout has no room for a sequence shorter than the window, and only the device
+    knows the lengths: every kernel that addresses scores leaves such a batch alone, the status
+    word says why, and nothing is written (the outputs keep their fill)."""
+    cfg = get_config("mistral7b_ragged").scaled(seq_lens=(900, 40), n_layers=2, budget_per_head=128)
+    q, k, v, cu = upload_model(cfg)
+    plan = make_plan(cfg, q, k, v, cu)
+    plan.scores.fill_(-7.0)
+    plan.keep_idx.fill_(-7)
+    plan.k_out.fill_(3.0)
+    lava.evict_model(plan, q, k, v)
+    assert lava.lava_poll_status(plan.workspace) & 1            # LAVA_DEV_SHORT_SEQUENCE
+    # (query groups scored as two halves start from a cleared score array: zeros, not the fill)
+    assert bool(((plan.scores == -7.0) | (plan.scores == 0.0)).all()) and bool((plan.keep_idx == -7).all())
+    assert bool((plan.k_out == 3.0).all())
+    cas = lava.Cascade(plan.desc, cfg.n_layers, sum(cfg.total_budget(b) for b in range(cfg.batch)),
+                       kv_dtype=k.dtype)
+    cas.begin(plan.total_budget)
+    for l in range(cfg.n_layers):
+        cas.step(q[l], k[l], v[l])
+    assert lava.lava_poll_status(cas.workspace) & 1
+    cas.close()
+    # the CUDA-core path (fp32) behaves the same
+    cfg = get_config("tiny").scaled(seq_lens=(300, 9), n_layers=1)
+    q, k, v, cu = upload_model(cfg)
+    plan = make_plan(cfg, q, k, v, cu)
+    plan.scores.fill_(-7.0)
+    lava.evict_model(plan, q, k, v)
+    assert lava.lava_poll_status(plan.workspace) & 1
+    assert bool((plan.scores == -7.0).all())

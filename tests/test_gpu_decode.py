@@ -80,3 +80,23 @@ def test_decode_attention_reads_a_cascade_state():
     torch.cuda.synchronize()
     _check(cfg, q_new, view["k_out"], view["v_out"], view["head_offsets"], view["layer_row_offset"], out, L)
     cas.close()
+
+
+def test_decode_attention_with_eight_queries_per_kv_head():
+    """G = 8 fills the eight real rows of the padded query operand; w = 16 keeps the score path
+    on one unit."""
+    cfg = get_config("llama8b_8k").scaled(seq_lens=(1500,), n_layers=2, n_q_heads=32, n_kv_heads=4,
+                                          window=16, budget_per_head=300)
+    q, k, v, cu = upload_model(cfg)
+    L = cfg.n_layers
+    plan = make_plan(cfg, q, k, v, cu)
+    lava.evict_model(plan, q, k, v)
+    assert lava.lava_poll_status(plan.workspace) == 0
+    gen = torch.Generator().manual_seed(23)
+    q_new = torch.randn(L, 1, cfg.n_q_heads, cfg.head_dim, generator=gen).to(k.dtype).cuda()
+    out = torch.empty((L, 1, cfg.n_q_heads, cfg.head_dim), device="cuda")
+    ws = torch.empty(lava.lava_decode_workspace_bytes(plan.desc, L), dtype=torch.uint8, device="cuda")
+    lava.lava_decode_attention_layers(plan.desc, L, q_new, plan.k_out, plan.v_out, plan.head_offsets,
+                                      plan.layer_row_offset, out, ws)
+    torch.cuda.synchronize()
+    _check(cfg, q_new, plan.k_out, plan.v_out, plan.head_offsets, plan.layer_row_offset, out, L)

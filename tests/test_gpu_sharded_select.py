@@ -23,7 +23,7 @@ def _desc(hkv, lens, w, cu):
 @pytest.mark.parametrize("ranks,hkv,lens,w,L", [
     (2, 8, (3000,), 32, 2),
     (4, 8, (2100, 700, 40), 32, 2),          # ragged batch, one sequence barely above the window
-    (2, 4, (9000, 20), 32, 1),               # a sequence shorter than the window: nothing to select
+    (2, 4, (9000, 32), 32, 1),               # a sequence of exactly the window: nothing to select
 ])
 def test_sharded_select_equals_the_unsplit_selection(ranks, hkv, lens, w, L):
     rng = np.random.RandomState(ranks * 100 + hkv)

@@ -6,8 +6,8 @@ LAVA_DEV_WAIT_EXPIRED, lava_poll_status must turn that into LAVA_ERR_TIMEOUT, an
 with the normal limit, on the same workspace, must be correct again.  (Waits for copies that are
 already in flight keep their long limit, so no CTA leaves under a running copy.)
 
-A sequence shorter than the window is scored as far as it goes and flagged with
-LAVA_DEV_SHORT_SEQUENCE on both score paths.
+A batch with a sequence shorter than the window has no room in the score layout: both score
+paths flag it with LAVA_DEV_SHORT_SEQUENCE and write nothing.
 """
 import numpy as np
 import pytest
@@ -70,24 +70,16 @@ def test_short_sequence_sets_the_status_bit(generic):
     lava.lava_set_option("force_generic", generic)
     try:
         assert lava.lava_score_path(desc) == (0 if generic else 1)
-        # total_scores counts n - w entries per sequence; the short one contributes none, so the
-        # array is sized for the two long sequences by hand
         w, hkv = cfg.window, cfg.n_kv_heads
-        sc = torch.zeros(hkv * (cfg.total_tokens - 3 * w) + 4096, dtype=torch.float32, device="cuda")
+        sc = torch.full((hkv * (cfg.total_tokens - 3 * w),), -7.0, dtype=torch.float32, device="cuda")
         vb = torch.zeros((3, hkv), dtype=torch.float32, device="cuda")
         ent = torch.zeros(3, dtype=torch.float64, device="cuda")
         lava.lava_score_layer(desc, q[0], k[0], v[0], None, sc, vb, ent, ws)
         status = lava.lava_poll_status(ws)
         assert status & LAVA_DEV_SHORT_SEQUENCE
         assert not status & LAVA_DEV_WAIT_EXPIRED
-        # A short sequence has no room in the score layout (its n - w is negative), so the arrays
-        # of its neighbours overlap by H_kv * (w - n) entries: that is why the call is flagged.
-        # What lies below the overlap, KV heads 0..6 of the first sequence, is still exact.
-        want = O.lava_scores(to_numpy64(q[0, 0]), to_numpy64(k[0, :, :700]), to_numpy64(v[0, :, :700]),
-                             w, cfg.pool_kind, cfg.pool_kernel)
-        got = sc[: hkv * (700 - w)].cpu().numpy().reshape(want.shape).astype(np.float64)
-        assert (hkv - 1) * (700 - w) <= hkv * (700 + 20 - 2 * w)
-        assert np.all(np.abs(got[:hkv - 1] - want[:hkv - 1])
-                      <= SCORE_RTOL * np.abs(want[:hkv - 1]) + SCORE_ATOL)
+        # The short sequence's n - w is negative, so its neighbours' score arrays would overlap and
+        # the last one would run past the end of the layer: nothing may be written.
+        assert bool((sc == -7.0).all())
     finally:
         lava.lava_set_option("force_generic", 0)
